@@ -1,0 +1,417 @@
+"""Benchmark of the PoT hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+One "step" = one decode token through the linear layers of a Llama-2-7B-shaped model
+(32 layers x {qkv 4096->12288, o 4096->4096, gate 4096->11008, up 4096->11008, down 11008->4096}):
+160 fused dequant+GEMV launches over 3-bit, group-128 PoT codes (2.53 GB of codes + scales, so
+every step streams its weights from HBM: the inputs are ~20x larger than L2).  The metric is the
+achieved algorithmic GB/s (codes + scales + x + y bytes per step / step time).  The same JSON
+line carries: the 2-bit chain, the standalone dequant throughput next to the uniform-INT twin,
+the small-batch and prefill GEMM figures, the roofline fraction of the dominant kernel, the
+oracle timed on the host cores, and an end-to-end figure with activations/results in host memory.
+
+With --gpus N > 1 (launched by torch.distributed.run) every rank runs its own replica of the
+chain (the path needs no exchange step); the value is the sum over ranks / max time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2507_11959_b200 import synth  # noqa: E402
+
+METRIC = "pot_dequant_gemv_GBps"
+UNIT = "GB/s"
+GROUP = 128
+HEADLINE_BITS = 3
+
+
+def gemv_bytes(N, K, bits, G, M=1):
+    return N * K * bits // 8 + N * (K // G) * 2 + 2 * K * M + 2 * N * M
+
+
+def read_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def reference_arm(args):
+    """The CPU oracle, as it stands, timed on the host cores on a bounded sample of the workload:
+    each step = the five projections of ONE layer of the chain (202 M weights), 3-bit, group 128."""
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    from oracle import pot_oracle as oracle
+    layer, nbytes = [], 0
+    for i, pr in enumerate(synth.LLAMA2_7B):
+        W = synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5")
+        codes, S = oracle.quantize(W, HEADLINE_BITS, GROUP, oracle.RULE_TOP)
+        x = synth.activations(synth.rng_for(2, 2 * i + 1), 1, pr.K)
+        layer.append((oracle.pack(codes, HEADLINE_BITS), S, pr.K, x))
+        nbytes += gemv_bytes(pr.N, pr.K, HEADLINE_BITS, GROUP)
+        del W, codes
+
+    def step():
+        for packed, S, K, x in layer:
+            oracle.matmul(packed, S, K, HEADLINE_BITS, GROUP, x)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = nbytes / dt / 1e9
+    sample = "one layer (5 projections, 202M weights) of the 32-layer chain per step, FP64 GEMV from packed codes"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama2-7b-shaped decode chain, batch 1, PoT 3-bit g128 (bounded sample: 1 of 32 layers per step)"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-config tables (chain only)")
+    ap.add_argument("--layers", type=int, default=synth.LLAMA2_7B_LAYERS)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    from paper_2507_11959_b200 import binding as B
+    from paper_2507_11959_b200 import dist as pdist
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    rank, local_rank, world = pdist.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.lib()
+    peaks = read_peaks()
+    stream = torch.cuda.Stream(device=dev)
+
+    def f16(bits16):
+        return torch.from_numpy(bits16.view(np.int16)).view(torch.float16).to(dev)
+
+    # ---- build the chain: one layer of seeded weights, quantized on the device, replicated per layer
+    def build_chain(bits):
+        protos = []
+        for i, pr in enumerate(synth.LLAMA2_7B):
+            W = f16(synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5"))
+            packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
+            tiled = B.pot_repack(packed, pr.K, bits, 0)
+            x = f16(synth.activations(synth.rng_for(2, 2 * i + 1), 1, pr.K)[0])
+            y = torch.empty(pr.N, dtype=torch.float16, device=dev)
+            ws_bytes = B.pot_gemv_workspace_bytes(pr.N, pr.K, bits, GROUP)
+            ws = B.new_workspace(ws_bytes, dev)
+            protos.append((pr, tiled, S, x, y, ws))
+            del W, packed
+        layers = []
+        for _ in range(args.layers):  # distinct buffers per layer: the chain streams from HBM
+            layers.append([(pr, t.clone(), s.clone(), x, y, ws) for (pr, t, s, x, y, ws) in protos])
+        nbytes = args.layers * sum(gemv_bytes(pr.N, pr.K, bits, GROUP) for pr in synth.LLAMA2_7B)
+        return layers, nbytes
+
+    def enqueue_chain(layers, bits, s):
+        for layer in layers:
+            for pr, t, sc, x, y, ws in layer:
+                B.pot_gemv(t, sc, pr.K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s)
+
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn(stream)  # warm-up outside capture
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                fn(stream)
+        return g
+
+    def time_graph(g, steps, warmup):
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                g.replay()
+            stream.synchronize()
+            pdist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            torch.cuda.synchronize()
+            pdist.barrier()
+        return e0.elapsed_time(e1) / steps  # ms per step
+
+    layers3, bytes3 = build_chain(HEADLINE_BITS)
+    launches_before = B.pot_launch_count()
+    g3 = capture(lambda s: enqueue_chain(layers3, HEADLINE_BITS, s))
+    launches_per_step = (B.pot_launch_count() - launches_before) // 2
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    ms = time_graph(g3, args.steps, args.warmup)
+    clocks = sampler.stop()
+    ms = pdist.max_over_ranks(ms, dev)
+    value = world * bytes3 / (ms * 1e-3) / 1e9
+
+    # ---- end to end: activations and results in pinned host memory, weights resident
+    host = []
+    for pr, t, sc, x, y, ws in layers3[0]:
+        xh = torch.empty(pr.K, dtype=torch.float16).pin_memory()
+        xh.copy_(x.cpu())
+        yh = torch.empty(pr.N, dtype=torch.float16).pin_memory()
+        host.append((xh, yh))
+
+    def enqueue_e2e(s):
+        for layer in layers3:
+            for (pr, t, sc, x, y, ws), (xh, yh) in zip(layer, host):
+                B.pot_gemv_host(t, sc, pr.K, HEADLINE_BITS, GROUP, xh, yh, x, y, B.TILED, workspace=ws, stream=s)
+
+    ge = capture(enqueue_e2e)
+    ms_e2e = pdist.max_over_ranks(time_graph(ge, max(3, args.steps // 2), 3), dev)
+    h2d = args.layers * sum(2 * pr.K for pr in synth.LLAMA2_7B)
+    d2h = args.layers * sum(2 * pr.N for pr in synth.LLAMA2_7B)
+    e2e = {"value": world * bytes3 / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": ms_e2e, "note": "x from pinned host and y to pinned host for each of the 160 GEMVs; weights resident in HBM"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 (int32 bit ops, f32 accumulate)",
+        "data": "synthetic",
+        "config": {"workload": f"llama2-7b-shaped decode chain, batch 1, {args.layers} layers x 5 projections, PoT {HEADLINE_BITS}-bit g{GROUP}, tiled layout, CUDA graph + PDL",
+                   "l2": "inputs larger than L2 (%.2f GB of codes+scales per step vs 126 MB)" % (bytes3 / 1e9),
+                   "bytes_per_step": bytes3, "launches_per_step": launches_per_step},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": value / world / peaks["hbm_gbs"], "frac_of_8TBs_nominal": value / world / 8000.0,
+                     "peak_source": peaks["source"], "kernel": "gemv_tiled_kernel<3,false>",
+                     "traffic": None},
+    }
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        out["extras"] = extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_chain, enqueue_chain)
+        out["cpu_baseline"] = cpu_baseline()
+    del layers3
+    if rank == 0:
+        print(json.dumps(out))
+
+
+def cpu_baseline():
+    """The oracle's FP64 GEMV from packed codes on the host cores: one layer of the chain (bounded sample)."""
+    from oracle import pot_oracle as oracle
+    layer, nbytes = [], 0
+    for i, pr in enumerate(synth.LLAMA2_7B):
+        W = synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5")
+        codes, S = oracle.quantize(W, HEADLINE_BITS, GROUP, oracle.RULE_TOP)
+        layer.append((oracle.pack(codes, HEADLINE_BITS), S, pr.K, synth.activations(synth.rng_for(2, 2 * i + 1), 1, pr.K)))
+        nbytes += gemv_bytes(pr.N, pr.K, HEADLINE_BITS, GROUP)
+    best = 1e30
+    for _ in range(3):
+        t0 = time.perf_counter()
+        for packed, S, K, x in layer:
+            oracle.matmul(packed, S, K, HEADLINE_BITS, GROUP, x)
+        best = min(best, time.perf_counter() - t0)
+    return {"value": nbytes / best / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "one layer (5 projections, 202M weights) of the 32-layer chain, best of 3"}
+
+
+def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_chain, enqueue_chain):
+    """Per-config tables: 2-bit chain, per-projection GEMV, dequant sweep vs the uniform twin, small-batch and prefill GEMM."""
+    ex = {}
+    hbm = peaks["hbm_gbs"]
+
+    # 2-bit chain (config 2)
+    layers2, bytes2 = build_chain(2)
+    g2 = capture(lambda s: enqueue_chain(layers2, 2, s))
+    ms2 = time_graph(g2, max(5, args.steps // 2), 3)
+    ex["chain_2bit"] = {"GBps": bytes2 / ms2 / 1e6, "ms_per_step": ms2, "frac_of_measured_hbm": bytes2 / ms2 / 1e6 / hbm}
+    del g2, layers2
+    torch.cuda.empty_cache()
+
+    def rotating(make, copies):
+        return [make() for _ in range(copies)]
+
+    # per-projection GEMV, HBM-cold (rotating copies > 4x L2), PoT vs uniform twin, tiled layout, + config 1
+    rows = []
+    shapes = [("cfg1 4096x4096", 4096, 4096, "normal")] + [(f"7B {p.name}", p.N, p.K, "t5") for p in synth.LLAMA2_7B if p.name != "up"]
+    for name, N, K, dist in shapes:
+        W = f16(synth.weights(synth.rng_for(1, N % 97), N, K, dist))
+        x = f16(synth.activations(synth.rng_for(1, 1 + N % 97), 1, K)[0])
+        y = torch.empty(N, dtype=torch.float16, device=dev)
+        for bits in (2, 3, 4):
+            packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
+            tiled = B.pot_repack(packed, K, bits, 0)
+            up, uS, uZ = B.uint_quantize_ref(W, bits, GROUP)
+            utiled = B.uint_repack(up, K, bits, 0)
+            copies = max(2, int(4 * 126e6 / (N * K * bits / 8)) + 1)
+            ws = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, bits, GROUP), dev)
+            pts = [(tiled.clone(), S.clone()) for _ in range(copies)]
+            uts = [(utiled.clone(), uS.clone(), uZ.clone()) for _ in range(copies)]
+            gp = capture(lambda s: [B.pot_gemv(t, sc, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s) for t, sc in pts])
+            gu = capture(lambda s: [B.uint_gemv(t, sc, z, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s) for t, sc, z in uts])
+            tp = min(time_graph(gp, 10, 3) for _ in range(3)) / copies
+            tu = min(time_graph(gu, 10, 3) for _ in range(3)) / copies
+            bp = gemv_bytes(N, K, bits, GROUP)
+            bu = bp + N * (K // GROUP) * 2
+            rows.append({"shape": name, "bits": bits, "pot_us": tp * 1e3, "pot_GBps": bp / tp / 1e6, "pot_frac_hbm": bp / tp / 1e6 / hbm,
+                         "uint_us": tu * 1e3, "uint_GBps": bu / tu / 1e6, "pot_speedup_vs_uint": tu / tp})
+            del pts, uts, gp, gu
+        del W
+        torch.cuda.empty_cache()
+    ex["gemv_per_projection_hbm_cold"] = rows
+
+    # standalone dequant (config 3): PoT vs uniform twin (fast and naive), FP16 out
+    rows = []
+    for N, K in synth.DEQUANT_SWEEP:
+        W = f16(synth.weights(synth.rng_for(3, N % 89), N, K, "normal"))
+        out = torch.empty((N, K), dtype=torch.float16, device=dev)
+        for bits in (2, 3, 4):
+            for G in (64, 128):
+                packed, S = B.pot_quantize_ref(W, bits, G, B.SCALE_TOP)
+                up, uS, uZ = B.uint_quantize_ref(W, bits, G)
+                reps = max(1, int(2e9 / (N * K * 2.4)))
+                gp = capture(lambda s: [B.pot_dequant(packed, S, K, bits, G, B.F16, out=out, stream=s) for _ in range(reps)])
+                gf = capture(lambda s: [B.uint_dequant(up, uS, uZ, K, bits, G, B.UINT_FAST, out=out, stream=s) for _ in range(reps)])
+                gn = capture(lambda s: [B.uint_dequant(up, uS, uZ, K, bits, G, B.UINT_NAIVE, out=out, stream=s) for _ in range(reps)])
+                tp, tf, tn = [min(time_graph(g, 5, 3) for _ in range(3)) / reps for g in (gp, gf, gn)]
+                nb = N * K * bits // 8 + N * (K // G) * 2 + N * K * 2
+                rows.append({"N": N, "K": K, "bits": bits, "G": G, "pot_us": tp * 1e3, "pot_Gweights_s": N * K / tp / 1e6,
+                             "pot_GBps": nb / tp / 1e6, "pot_frac_hbm": nb / tp / 1e6 / hbm, "uint_fast_us": tf * 1e3,
+                             "uint_naive_us": tn * 1e3, "pot_speedup_vs_best_uint": min(tf, tn) / tp})
+                del gp, gf, gn
+        del W, out
+        torch.cuda.empty_cache()
+    ex["dequant_sweep"] = rows
+
+    # small-batch GEMM (config 4), HBM-cold
+    rows = []
+    for pr in synth.LLAMA2_13B:
+        W = f16(synth.weights(synth.rng_for(4, pr.N % 83), pr.N, pr.K, "t5"))
+        packed, S = B.pot_quantize_ref(W, 3, GROUP, B.SCALE_TOP)
+        tiled = B.pot_repack(packed, pr.K, 3, 0)
+        copies = max(2, int(4 * 126e6 / (pr.N * pr.K * 3 / 8)) + 1)
+        pts = [(tiled.clone(), S.clone()) for _ in range(copies)]
+        del W, packed
+        for M in synth.SMALL_BATCH_M:
+            X = f16(synth.activations(synth.rng_for(4, 7), M, pr.K))
+            Y = torch.empty((M, pr.N), dtype=torch.float16, device=dev)
+            ws = B.new_workspace(B.pot_gemm_workspace_bytes(M, pr.N, pr.K, 3, GROUP), dev)
+            g = capture(lambda s: [B.pot_gemm(t, sc, pr.K, 3, GROUP, X, B.TILED, Y=Y, workspace=ws, stream=s) for t, sc in pts])
+            t = min(time_graph(g, 10, 3) for _ in range(3)) / copies
+            nb = gemv_bytes(pr.N, pr.K, 3, GROUP, M)
+            rows.append({"shape": f"13B {pr.name} {pr.K}->{pr.N}", "M": M, "us": t * 1e3, "GBps": nb / t / 1e6, "frac_hbm": nb / t / 1e6 / hbm})
+            del g
+        del pts
+        torch.cuda.empty_cache()
+    ex["small_batch_gemm"] = rows
+
+    # prefill GEMM (config 5)
+    rows = []
+    for pr in synth.LLAMA2_70B:
+        W = f16(synth.weights(synth.rng_for(5, pr.N % 79), pr.N, pr.K, "normal", 0.015))
+        X = f16(synth.activations(synth.rng_for(5, 5), synth.PREFILL_M, pr.K, outliers=False))
+        Y = torch.empty((synth.PREFILL_M, pr.N), dtype=torch.float16, device=dev)
+        for bits in (2, 3):
+            packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
+            layout, P = B.CANONICAL, packed
+            try:
+                tiled = B.pot_repack(packed, pr.K, bits, 0)
+                ws = B.new_workspace(B.pot_gemm_workspace_bytes(synth.PREFILL_M, pr.N, pr.K, bits, GROUP), dev)
+                B.pot_gemm(tiled, S, pr.K, bits, GROUP, X, B.TILED, Y=Y, workspace=ws, stream=stream)
+                layout, P = B.TILED, tiled
+            except B.PotError:
+                ws = None
+            g = capture(lambda s: B.pot_gemm(P, S, pr.K, bits, GROUP, X, layout, Y=Y, workspace=ws, stream=s))
+            t = min(time_graph(g, 3, 3) for _ in range(2))
+            fl = 2.0 * synth.PREFILL_M * pr.N * pr.K
+            rows.append({"shape": f"70B {pr.name} {pr.K}->{pr.N}", "M": synth.PREFILL_M, "bits": bits, "ms": t,
+                         "TFLOPs": fl / t / 1e9, "frac_tensor_sustained": fl / t / 1e9 / peaks["bf16_tflops_sustained"],
+                         "kernel": "tcgen05" if layout == B.TILED else "mma.sync fallback"})
+            del g
+        del W, X, Y
+        torch.cuda.empty_cache()
+    ex["prefill_gemm"] = rows
+    return ex
+
+
+if __name__ == "__main__":
+    main()

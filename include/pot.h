@@ -1,0 +1,198 @@
+/*
+ * pot.h -- C ABI of the B200 (sm_100a) PoT-PTQ inference library.
+ *
+ * The library implements the inference hot path of PoT-PTQ: n-bit power-of-two weight codes
+ * (one sign bit + an (n-1)-bit exponent E, one FP16 scale S per group of G weights along the
+ * reduction dimension) are unpacked to FP16/BF16 with integer bit manipulation and either
+ * stored (pot_dequant) or consumed directly by a GEMV / GEMM.
+ *
+ * Notation (paper, Sec. 3.1): W is [N, K] row-major, N = output features, K = input features
+ * (the reduction dimension); y = W x.  Groups are G contiguous elements of a row.
+ * q_max = 2^(n-1) - 1.  A code is  sign << (n-1) | E  (the paper's "S0 E1 E2" for n = 3).
+ *
+ * General conventions
+ *   - Unless a parameter is marked HOST, every data pointer is a DEVICE pointer owned by the
+ *     caller.  The library allocates nothing, keeps no per-call state and never synchronises;
+ *     every call enqueues its work on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and returns.
+ *   - Argument errors are detected on the host and returned BEFORE anything is launched.
+ *     POT_ERR_CUDA reports a failed launch.  Kernels never trap.
+ *   - Base pointers must be 16-byte aligned.  K % 128 == 0 and K % G == 0, bits in {2,3,4},
+ *     G in {64,128}.  (K % 128 == 0 makes every packed row a multiple of 16 bytes.)
+ *   - Scale contract: every scale is a normal FP16 number whose exponent field e satisfies
+ *     1 <= e and e + q_max <= 30, i.e. S in [2^-14, (2 - 2^-10) * 2^(15 - q_max)].  Inside that
+ *     range adding E to the exponent field is exactly multiplication by 2^E; outside it
+ *     (zero, subnormal, too large) the results are unspecified but no call faults.
+ *     pot_quantize_ref never produces an illegal scale; pot_validate_scales counts them.
+ *
+ * Interchange ("canonical") layout of the codes -- the paper does not specify one:
+ *   row i is a little-endian bit stream of K*n/8 bytes; code k occupies bits [n*k, n*k+n)
+ *   counted from the least significant bit of byte 0.  Example, n = 3: codes
+ *   011,101,000,111,000,010,100,000 -> bytes 2B 0E 11.   Scales: [N, K/G] row-major FP16.
+ *
+ * Kernel ("tiled") layout, produced by pot_repack: a size-preserving bijection of the same
+ * bits (exactly n bits per weight, no padding) that lets a warp fetch the codes of a
+ * 16-row x 128-column block with fully coalesced 16-byte loads and place two weights in a
+ * 32-bit lane with one mask and one shift-add.  It requires N % 16 == 0.  See pot_repack.
+ */
+#ifndef POT_B200_H
+#define POT_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    POT_OK = 0,
+    POT_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+    POT_ERR_UNSUPPORTED = 2, /* bits not in {2,3,4}, G not in {64,128}, unknown enum value   */
+    POT_ERR_SHAPE = 3,       /* N, M <= 0; K % 128 != 0; K % G != 0; tiled layout with N % 16 */
+    POT_ERR_ALIGN = 4,       /* a base pointer is not 16-byte aligned                        */
+    POT_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than the *_workspace_bytes value   */
+    POT_ERR_SCALE_RANGE = 6, /* reserved for callers that act on pot_validate_scales          */
+    POT_ERR_CUDA = 7         /* the CUDA runtime reported an error for this call's launch     */
+} pot_status_t;
+
+typedef enum { POT_F16 = 0, POT_BF16 = 1 } pot_dtype_t;
+
+/* How pot_quantize_ref chooses the group scale (paper: scale search is Algorithm 1). */
+typedef enum {
+    POT_SCALE_TOP = 0,      /* S = max|w| * 2^-q_max : the top level 2^q_max * S sits on max|w| */
+    POT_SCALE_PAPER_S0 = 1, /* S = fp16(max|w| / (2^q_max - 1)) : Algorithm 1's s0 with b = 1   */
+    POT_SCALE_GIVEN = 2,    /* S is supplied by the caller (must satisfy the scale contract)    */
+    POT_SCALE_SEARCH = 3    /* S = s0 * b*, b* from Algorithm 1's 200-point grid search          */
+} pot_scale_rule_t;
+
+typedef enum { POT_LAYOUT_CANONICAL = 0, POT_LAYOUT_TILED = 1 } pot_layout_t;
+
+/* Which uniform-INT dequantization kernel to run (same result, bit for bit). */
+typedef enum {
+    UINT_KERNEL_FAST = 0,  /* packed-half arithmetic: integer -> FP16 by exponent splicing, HSUB2, HMUL2 */
+    UINT_KERNEL_NAIVE = 1  /* per-element int -> float convert, subtract, multiply, convert back  */
+} uint_kernel_t;
+
+const char* pot_status_string(pot_status_t s);
+
+/* ---- sizes (host arithmetic only; 0 on invalid arguments) ------------------------------- */
+size_t pot_packed_bytes(int64_t N, int64_t K, int bits);          /* N * K * bits / 8          */
+size_t pot_scales_bytes(int64_t N, int64_t K, int group);         /* N * (K / group) * 2       */
+/* Scratch needed by pot_gemv / uint_gemv with the tiled layout (split-K arrival counters +
+ * FP32 partial sums); may be 0.  The workspace must be ZERO before its first use; every call
+ * leaves the counters at zero again, so one buffer can serve all calls on one stream.  Two
+ * calls that may run concurrently (different streams) need different workspaces.            */
+size_t pot_gemv_workspace_bytes(int64_t N, int64_t K, int bits, int group);
+/* Scratch needed by pot_gemm for the given M; may be 0.                                       */
+size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group);
+
+/* Number of kernels this process has launched through the library (diagnostic counter). */
+uint64_t pot_launch_count(void);
+
+/*
+ * pot_quantize_ref -- reference PoT quantizer (Eq. 2; groups per Sec. 3.1).  Set-up code: it
+ * makes the inputs of the hot path and is not part of the timed path.
+ *   W_f16      [N,K] FP16, finite values.
+ *   scales_f16 [N,K/G] FP16: read when rule == POT_SCALE_GIVEN, written otherwise (after
+ *              clamping into the legal scale range; an all-zero group gets 2^-14).
+ *   packed_out [N, K*bits/8] canonical layout.
+ * Per weight: sign = [w < 0] (so -0 -> +), E = clamp(round(log2(|w|/S)), 0, q_max), evaluated
+ * exactly (threshold test on w^2 against 2^(2k+1) S^2 in FP64; |w| = 0 gives E = 0).
+ */
+pot_status_t pot_quantize_ref(const void* W_f16, int64_t N, int64_t K, int bits, int group,
+                              pot_scale_rule_t rule, void* scales_f16, void* packed_out, void* stream);
+
+/*
+ * pot_validate_scales -- counts scales outside the scale contract.
+ *   d_bad_count: device int32; the kernel ADDS the number of offending entries (zero it first).
+ */
+pot_status_t pot_validate_scales(const void* scales_f16, int64_t count, int bits, int32_t* d_bad_count,
+                                 void* stream);
+
+/*
+ * pot_repack -- canonical -> tiled (direction 0) or tiled -> canonical (direction 1).
+ * Both buffers hold pot_packed_bytes(N,K,bits) bytes and must not overlap.  N % 16 == 0.
+ *
+ * Tiled layout: the matrix is cut into units of 16 rows x 128 columns (one unit per row block
+ * rb = i/16 and column block cb = k/128, stored in [rb][cb] order, 16*128*n/8 bytes each).
+ * A unit holds n "planes" of 256 bytes; plane t stores, for row r of the unit, the 16-byte
+ * word t of that row's 128-code record at byte offset t*256 + r*16.  The record of one row
+ * (n 16-byte words = 4n 32-bit words) arranges its 128 codes so that codes 2p and 2p+1 of an
+ * 8-code block sit 16 bits apart in one 32-bit word (see csrc/layout.cuh for the bit map).
+ */
+pot_status_t pot_repack(const void* src, void* dst, int64_t N, int64_t K, int bits, int direction,
+                        void* stream);
+
+/* Host arithmetic only: position (32-bit word index inside the 4n-word record, bit index) of
+ * bit b of code q (0 <= q < 128) in the tiled layout.  kind 0 = PoT codes, 1 = uniform codes. */
+pot_status_t pot_layout_bit(int bits, int kind, int q, int b, int* word, int* bit);
+
+/*
+ * pot_dequant -- the paper's dequantization kernel (Sec. 4.2): extract the exponent field with
+ * an AND mask, move the sign to bit 15, OR them, align to the FP16 exponent (bit 10; bit 7 for
+ * BF16) and integer-add to the scale's bit pattern.  No floating-point instruction touches the
+ * weights.  packed is canonical; W_out is [N,K] row-major of out_dtype (2 bytes per element).
+ * BF16: the FP16 scale is converted once per group to BF16 (round to nearest even).
+ */
+pot_status_t pot_dequant(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                         int group, pot_dtype_t out_dtype, void* W_out, void* stream);
+
+/*
+ * pot_gemv -- batch-1 decode: y = W~ x with W~ the FP16 reconstruction (Eq. 1), FP32
+ * accumulation, FP16 output.  CUDA-core kernel: codes are decoded in registers with the
+ * integer-add trick, lanes reduce over K with warp shuffles, and K is split across CTAs when N
+ * alone cannot fill the GPU (partials in `workspace`, summed in a fixed order, so results are
+ * bit-identical run to run).
+ *   x_f16 [K], y_f16 [N]; workspace >= pot_gemv_workspace_bytes(N,K,bits,group), 16-byte aligned
+ *   (may be NULL when that size is 0).  `layout` says how `packed` is arranged.
+ */
+pot_status_t pot_gemv(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                      int group, pot_layout_t layout, const void* x_f16, void* y_f16,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pot_gemv_host -- pot_gemv for a caller whose activations and results live in HOST memory
+ * (ideally pinned): copies x_host [K] to d_x, runs pot_gemv, copies the result to y_host [N],
+ * all asynchronously on `stream`.  The weights stay resident on the device.
+ *   x_host, y_host: HOST pointers.  d_x (>= 2K bytes) and d_y (>= 2N bytes): device staging
+ *   buffers owned by the caller.  The caller synchronises the stream before reading y_host.
+ */
+pot_status_t pot_gemv_host(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                           int group, pot_layout_t layout, const void* x_host, void* y_host,
+                           void* d_x, void* d_y, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pot_gemm -- Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
+ * accumulation, FP16 output.  M <= 32 (decode batches) runs a bandwidth-bound tensor-core
+ * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the
+ * tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
+ * accumulators in tensor memory.  The prefill kernel requires layout == POT_LAYOUT_TILED.
+ */
+pot_status_t pot_gemm(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                      int group, pot_layout_t layout, const void* X_f16, int64_t M, void* Y_f16,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- uniform-INT (zero-point) twin at the same bits and group size ------------------------
+ * The baseline the paper compares against (first equation of Sec. 4.1): w~ = (W_Q + Z) o S.
+ * Here the stored zero-point z is non-negative (Z = -z): codes q in [0, 2^n - 1] in the same
+ * canonical bit-stream layout, scales_f16 and zeros_f16 [N,K/G] FP16 (zeros hold the integer z
+ * as an FP16 number, so storage is n + 32/G bits per weight).  w~ = fp16((q - z) * s): the
+ * integer difference is exact and the product is rounded once.
+ */
+pot_status_t uint_quantize_ref(const void* W_f16, int64_t N, int64_t K, int bits, int group,
+                               void* scales_f16, void* zeros_f16, void* packed_out, void* stream);
+pot_status_t uint_dequant(const void* packed, const void* scales_f16, const void* zeros_f16, int64_t N,
+                          int64_t K, int bits, int group, uint_kernel_t kernel, void* W_out_f16, void* stream);
+pot_status_t uint_gemv(const void* packed, const void* scales_f16, const void* zeros_f16, int64_t N,
+                       int64_t K, int bits, int group, pot_layout_t layout, const void* x_f16, void* y_f16,
+                       void* workspace, size_t workspace_bytes, void* stream);
+/* canonical <-> tiled for uniform codes (same unit/plane structure as pot_repack; the n-bit
+ * integer is kept as one field, see csrc/layout.cuh).  direction 0: canonical -> tiled.       */
+pot_status_t uint_repack(const void* src, void* dst, int64_t N, int64_t K, int bits, int direction,
+                         void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POT_B200_H */

@@ -1,0 +1,86 @@
+// Shared host/device helpers of the PoT library: argument checks, launch bookkeeping,
+// canonical-layout field extraction.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "../../include/pot.h"
+
+namespace pot {
+
+extern std::atomic<uint64_t> g_launches;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline pot_status_t check_shape(int64_t N, int64_t K, int bits, int group) {
+    if (bits < 2 || bits > 4) return POT_ERR_UNSUPPORTED;
+    if (group != 64 && group != 128) return POT_ERR_UNSUPPORTED;
+    if (N <= 0 || K <= 0) return POT_ERR_SHAPE;
+    if (K % 128 != 0 || K % group != 0) return POT_ERR_SHAPE;
+    if (N > (int64_t(1) << 31) || K > (int64_t(1) << 31)) return POT_ERR_SHAPE;
+    return POT_OK;
+}
+
+// Call after a kernel launch: counts it and maps a launch error to a status.
+inline pot_status_t launched(int n = 1) {
+    g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? POT_OK : POT_ERR_CUDA;
+}
+
+constexpr int kSmCount = 148;  // B200: 2 dies x 74 SMs
+
+#ifdef __CUDACC__
+// Launch with programmatic stream serialization: the kernel may start while the previous kernel
+// in the stream is still draining; it must execute griddepcontrol.wait before touching anything
+// the previous kernel wrote (and before writing anything the previous kernel may still read).
+template <typename... Args>
+inline pot_status_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args...);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return e == cudaSuccess ? POT_OK : POT_ERR_CUDA;
+}
+#endif
+
+#ifdef __CUDACC__
+__host__ __device__ constexpr int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
+
+// Read `nbits` (<= 32) bits starting at bit offset `bitoff` of a little-endian bit stream whose
+// 32-bit words are `p` (4-byte aligned).  The second word is read only when the field spills.
+__device__ __forceinline__ uint32_t read_bits(const uint32_t* __restrict__ p, int64_t bitoff, int nbits) {
+    const int64_t w = bitoff >> 5;
+    const int sh = (int)(bitoff & 31);
+    uint32_t lo = __ldg(p + w);
+    uint32_t hi = (sh + nbits > 32) ? __ldg(p + w + 1) : 0u;
+    uint32_t v = __funnelshift_r(lo, hi, sh);
+    return nbits == 32 ? v : (v & ((1u << nbits) - 1u));
+}
+
+// Sec. 4.2, stage 1 on one canonical code c = sign << (n-1) | E:
+//   exponent bits by AND mask, sign moved to the top, OR  ->  [S | 0.. E] as a 6-bit word,
+//   aligned so that E sits at bit `ebit` (10 for FP16, 7 for BF16) and the sign at bit 15.
+template <int BITS>
+__device__ __forceinline__ uint32_t signed_exponent(uint32_t c, int ebit) {
+    const uint32_t e = (c & (uint32_t)qmax_of(BITS)) << ebit;
+    const uint32_t s = (c << (16 - BITS)) & 0x8000u;
+    return e | s;
+}
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
+}  // namespace pot

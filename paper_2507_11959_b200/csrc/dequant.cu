@@ -1,0 +1,182 @@
+// Standalone dequantization kernels: PoT (Sec. 4.2 of the paper) and the uniform-INT twin
+// (first equation of Sec. 4.1).  Both stream canonical codes + per-group FP16 parameters from
+// HBM and write [N,K] 16-bit weights; they are bound by HBM bandwidth (mostly the 2-byte
+// write per weight), so the work is laid out for full-width coalesced stores: consecutive
+// lanes produce consecutive 16-byte pieces of a row, and every thread has several independent
+// pieces in flight.
+#include "common.cuh"
+
+namespace pot {
+
+constexpr int DQ_THREADS = 256;
+constexpr int DQ_UNROLL = 4;  // 8-code pieces per thread
+
+// 8 canonical codes (8*BITS bits in v) -> 4 words with the code pairs spread 16 bits apart:
+// out[j] = code(2j) | code(2j+1) << 16
+template <int BITS>
+__device__ __forceinline__ void spread_pairs(uint32_t v, uint32_t (&out)[4]) {
+    constexpr uint32_t CM = (1u << BITS) - 1u;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t t = v >> (2 * j * BITS);
+        out[j] = (t & CM) | ((t << (16 - BITS)) & (CM << 16));
+    }
+}
+
+// PoT: FP16 (EBIT = 10) or BF16 (EBIT = 7) output.
+template <int BITS, int EBIT>
+__global__ void __launch_bounds__(DQ_THREADS) pot_dequant_kernel(const uint32_t* __restrict__ packed,
+                                                                 const uint16_t* __restrict__ scales, int64_t n_pieces,
+                                                                 int pieces_per_group, uint4* __restrict__ out) {
+    constexpr uint32_t QM2 = (uint32_t)qmax_of(BITS) * 0x10001u;   // exponent mask, both halves
+    constexpr uint32_t SM2 = (1u << (BITS - 1)) * 0x10001u;        // sign mask, both halves
+    const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
+    uint32_t v[DQ_UNROLL];
+    uint32_t sc[DQ_UNROLL];
+#pragma unroll
+    for (int u = 0; u < DQ_UNROLL; ++u) {
+        const int64_t c = base + (int64_t)u * DQ_THREADS;
+        if (c < n_pieces) {
+            v[u] = read_bits(packed, c * (8 * BITS), 8 * BITS);
+            sc[u] = __ldg(scales + c / pieces_per_group);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < DQ_UNROLL; ++u) {
+        const int64_t c = base + (int64_t)u * DQ_THREADS;
+        if (c >= n_pieces) continue;
+        uint32_t s16 = sc[u];
+        if (EBIT == 7) {  // BF16 output: round the FP16 scale once to BF16
+            s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
+        }
+        const uint32_t sc2 = s16 * 0x10001u;
+        uint32_t pr[4];
+        spread_pairs<BITS>(v[u], pr);
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            // stage 1 (bit manipulation): exponent by AND mask, sign moved up, OR;
+            // stage 2 (fixed-point add): align with the exponent field and add to the scale's bits.
+            const uint32_t signed_exp = ((pr[j] & QM2) << EBIT) | ((pr[j] & SM2) << (16 - BITS));
+            o[j] = sc2 + signed_exp;
+        }
+        out[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// uniform twin, packed-half arithmetic: q -> FP16 by splicing it under the exponent of 1024,
+// (1024 + q) - (1024 + z) is exact, one HMUL2 by the scale rounds once.
+template <int BITS>
+__global__ void __launch_bounds__(DQ_THREADS) uint_dequant_fast_kernel(const uint32_t* __restrict__ packed,
+                                                                       const uint16_t* __restrict__ scales,
+                                                                       const uint16_t* __restrict__ zeros,
+                                                                       int64_t n_pieces, int pieces_per_group,
+                                                                       uint4* __restrict__ out) {
+    const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
+    uint32_t v[DQ_UNROLL];
+    uint32_t sc[DQ_UNROLL], zp[DQ_UNROLL];
+#pragma unroll
+    for (int u = 0; u < DQ_UNROLL; ++u) {
+        const int64_t c = base + (int64_t)u * DQ_THREADS;
+        if (c < n_pieces) {
+            v[u] = read_bits(packed, c * (8 * BITS), 8 * BITS);
+            sc[u] = __ldg(scales + c / pieces_per_group);
+            zp[u] = __ldg(zeros + c / pieces_per_group);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < DQ_UNROLL; ++u) {
+        const int64_t c = base + (int64_t)u * DQ_THREADS;
+        if (c >= n_pieces) continue;
+        const __half2 s2 = __half2half2(__ushort_as_half((uint16_t)sc[u]));
+        const __half2 zm2 = __hadd2(__half2half2(__ushort_as_half((uint16_t)zp[u])), __float2half2_rn(1024.0f));
+        uint32_t pr[4];
+        spread_pairs<BITS>(v[u], pr);
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t h = pr[j] | 0x64006400u;  // half2{1024 + q0, 1024 + q1}
+            const __half2 d = __hsub2(*reinterpret_cast<const __half2*>(&h), zm2);
+            const __half2 w = __hmul2(d, s2);
+            o[j] = *reinterpret_cast<const uint32_t*>(&w);
+        }
+        out[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// uniform twin, the textbook form: integer -> float, subtract the zero-point, multiply by the scale.
+template <int BITS>
+__global__ void __launch_bounds__(DQ_THREADS) uint_dequant_naive_kernel(const uint32_t* __restrict__ packed,
+                                                                        const uint16_t* __restrict__ scales,
+                                                                        const uint16_t* __restrict__ zeros,
+                                                                        int64_t n_pieces, int pieces_per_group,
+                                                                        uint4* __restrict__ out) {
+    constexpr uint32_t CM = (1u << BITS) - 1u;
+    const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < DQ_UNROLL; ++u) {
+        const int64_t c = base + (int64_t)u * DQ_THREADS;
+        if (c >= n_pieces) continue;
+        const uint32_t v = read_bits(packed, c * (8 * BITS), 8 * BITS);
+        const float s = __half2float(__ushort_as_half(__ldg(scales + c / pieces_per_group)));
+        const float z = __half2float(__ushort_as_half(__ldg(zeros + c / pieces_per_group)));
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float q0 = (float)((v >> (2 * j * BITS)) & CM);
+            const float q1 = (float)((v >> ((2 * j + 1) * BITS)) & CM);
+            const __half2 w = __floats2half2_rn((q0 - z) * s, (q1 - z) * s);
+            o[j] = *reinterpret_cast<const uint32_t*>(&w);
+        }
+        out[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+}  // namespace pot
+
+using namespace pot;
+
+extern "C" pot_status_t pot_dequant(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                    pot_dtype_t out_dtype, void* W_out, void* stream) {
+    if (!packed || !scales || !W_out) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, bits, group);
+    if (st != POT_OK) return st;
+    if (out_dtype != POT_F16 && out_dtype != POT_BF16) return POT_ERR_UNSUPPORTED;
+    if (!aligned16(packed) || !aligned16(scales) || !aligned16(W_out)) return POT_ERR_ALIGN;
+    const int64_t n_pieces = N * K / 8;
+    const unsigned grid = (unsigned)((n_pieces + DQ_THREADS * DQ_UNROLL - 1) / (DQ_THREADS * DQ_UNROLL));
+    cudaStream_t s = (cudaStream_t)stream;
+    auto* P = (const uint32_t*)packed;
+    auto* S = (const uint16_t*)scales;
+    auto* O = (uint4*)W_out;
+    const int ppg = group / 8;
+#define POT_DQ(B)                                                                                     \
+    if (out_dtype == POT_F16) pot_dequant_kernel<B, 10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O); \
+    else pot_dequant_kernel<B, 7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
+    if (bits == 2) { POT_DQ(2) } else if (bits == 3) { POT_DQ(3) } else { POT_DQ(4) }
+#undef POT_DQ
+    return launched();
+}
+
+extern "C" pot_status_t uint_dequant(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
+                                     int bits, int group, uint_kernel_t kernel, void* W_out, void* stream) {
+    if (!packed || !scales || !zeros || !W_out) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, bits, group);
+    if (st != POT_OK) return st;
+    if (kernel != UINT_KERNEL_FAST && kernel != UINT_KERNEL_NAIVE) return POT_ERR_UNSUPPORTED;
+    if (!aligned16(packed) || !aligned16(scales) || !aligned16(zeros) || !aligned16(W_out)) return POT_ERR_ALIGN;
+    const int64_t n_pieces = N * K / 8;
+    const unsigned grid = (unsigned)((n_pieces + DQ_THREADS * DQ_UNROLL - 1) / (DQ_THREADS * DQ_UNROLL));
+    cudaStream_t s = (cudaStream_t)stream;
+    auto* P = (const uint32_t*)packed;
+    auto* S = (const uint16_t*)scales;
+    auto* Z = (const uint16_t*)zeros;
+    auto* O = (uint4*)W_out;
+    const int ppg = group / 8;
+#define UINT_DQ(B)                                                                                              \
+    if (kernel == UINT_KERNEL_FAST) uint_dequant_fast_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O); \
+    else uint_dequant_naive_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
+    if (bits == 2) { UINT_DQ(2) } else if (bits == 3) { UINT_DQ(3) } else { UINT_DQ(4) }
+#undef UINT_DQ
+    return launched();
+}
