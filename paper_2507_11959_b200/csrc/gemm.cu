@@ -68,6 +68,8 @@ __global__ void __launch_bounds__(GS_WARPS * 32) pot_gemm_small_kernel(const uin
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 
+    // Lanes whose column block lies beyond K (partial last chunk) keep all-zero records with scale 1.0
+    // and read x as zero: every lane of the warp must still execute the (warp-wide) MMA instructions.
     uint32_t rec[2][NW];
     uint32_t sc[2][2];
     auto load = [&](int chunk) {
@@ -85,6 +87,13 @@ __global__ void __launch_bounds__(GS_WARPS * 32) pot_gemm_small_kernel(const uin
                 sc[h][0] = (uint32_t)__ldg(sp) * 0x10001u;
                 sc[h][1] = (uint32_t)__ldg(sp + spr - 1) * 0x10001u;
             }
+        } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int i = 0; i < NW; ++i) rec[h][i] = 0u;
+                sc[h][0] = sc[h][1] = 0x3C003C00u;
+            }
         }
     };
     int c = chunk_begin + warp;
@@ -93,26 +102,25 @@ __global__ void __launch_bounds__(GS_WARPS * 32) pot_gemm_small_kernel(const uin
     pdl_wait();
     for (; c < chunk_end; c += GS_WARPS) {
         const int64_t cb = 4 * (int64_t)c + tig;
-        if (cb < ncb) {
+        const bool valid = cb < ncb;
 #pragma unroll
-            for (int blk = 0; blk < 8; ++blk) {
-                uint32_t w0[8], w1[8];
-                potl::pot_decode_pairs16<BITS>(rec[0], blk, sc[0][blk >> 2], w0);
-                potl::pot_decode_pairs16<BITS>(rec[1], blk, sc[1][blk >> 2], w1);
+        for (int blk = 0; blk < 8; ++blk) {
+            uint32_t w0[8], w1[8];
+            potl::pot_decode_pairs16<BITS>(rec[0], blk, sc[0][blk >> 2], w0);
+            potl::pot_decode_pairs16<BITS>(rec[1], blk, sc[1][blk >> 2], w1);
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const int token = 8 * mt + gid;
-                    uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
-                    if (token < M) {
-                        const uint4* xp = reinterpret_cast<const uint4*>(X + (int64_t)token * K + cb * 128) + 2 * blk;
-                        xa = __ldg(xp);
-                        xb = __ldg(xp + 1);
-                    }
-                    mma_16816(acc[mt], w0[0], w1[0], w0[1], w1[1], xa.x, xa.y);
-                    mma_16816(acc[mt], w0[2], w1[2], w0[3], w1[3], xa.z, xa.w);
-                    mma_16816(acc[mt], w0[4], w1[4], w0[5], w1[5], xb.x, xb.y);
-                    mma_16816(acc[mt], w0[6], w1[6], w0[7], w1[7], xb.z, xb.w);
+            for (int mt = 0; mt < MT; ++mt) {
+                const int token = 8 * mt + gid;
+                uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
+                if (valid && token < M) {
+                    const uint4* xp = reinterpret_cast<const uint4*>(X + (int64_t)token * K + cb * 128) + 2 * blk;
+                    xa = __ldg(xp);
+                    xb = __ldg(xp + 1);
                 }
+                mma_16816(acc[mt], w0[0], w1[0], w0[1], w1[1], xa.x, xa.y);
+                mma_16816(acc[mt], w0[2], w1[2], w0[3], w1[3], xa.z, xa.w);
+                mma_16816(acc[mt], w0[4], w1[4], w0[5], w1[5], xb.x, xb.y);
+                mma_16816(acc[mt], w0[6], w1[6], w0[7], w1[7], xb.z, xb.w);
             }
         }
         if (c + GS_WARPS < chunk_end) load(c + GS_WARPS);
