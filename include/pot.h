@@ -163,6 +163,29 @@ pot_status_t pot_gemv_host(const void* packed, const void* scales_f16, int64_t N
                            void* d_x, void* d_y, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * pot_gemv_noalloc -- pot_gemv (tiled layout) for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging convenience of this library.)
+ * Who needs it: a plug-in inside a host application that owns every byte of device memory and
+ * gives the plug-in no allocator -- for example an inference server whose serving loop may
+ * never run into the device-wide synchronisation that cudaMalloc / cudaFree imply.  Such a
+ * caller has nowhere to get the split-K workspace of pot_gemv from.  Here the workspace is a
+ * fixed array of pot_gemv_noalloc_max_scratch_bytes() = 1 MiB that is part of the library image:
+ * every GPU that loads the library holds it until the process exits.
+ *   - Arguments as for pot_gemv with layout = POT_LAYOUT_TILED; inputs and outputs are still the
+ *     caller's device buffers.  The call itself allocates and frees nothing.
+ *   - A shape whose workspace (pot_gemv_workspace_bytes) exceeds the array is rejected with
+ *     POT_ERR_WORKSPACE before anything is enqueued.
+ *   - The first call on each device (with that device current) looks the array's device address
+ *     up through the runtime.  Make that first call outside of any stream capture.
+ *   - All calls share the one array per GPU and it keeps the last call's contents; each call
+ *     clears the part that must start at zero on `stream`.  Calls that may overlap on the same
+ *     GPU (different streams) race on it -- serialise them, or use pot_gemv with own workspaces.
+ */
+size_t pot_gemv_noalloc_max_scratch_bytes(void);
+pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, int64_t N, int64_t K,
+                              int bits, int group, const void* x_f16, void* y_f16, void* stream);
+
+/*
  * pot_gemm -- Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
  * accumulation, FP16 output.  M <= 32 (decode batches) runs a bandwidth-bound tensor-core
  * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the

@@ -24,7 +24,7 @@ EXPORTS = [
     "pot_status_string", "pot_packed_bytes", "pot_scales_bytes", "pot_gemv_workspace_bytes",
     "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack",
     "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_host", "pot_gemm", "uint_quantize_ref", "uint_dequant",
-    "uint_gemv", "pot_layout_bit",
+    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes",
 ]
 
 _lib = None
@@ -66,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.uint_dequant.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.uint_gemv.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
         L.pot_layout_bit.argtypes = [i32, i32, i32, i32, vp, vp]
+        L.pot_gemv_noalloc.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp, vp]
+        L.pot_gemv_noalloc_max_scratch_bytes.restype = sz
+        L.pot_gemv_noalloc_max_scratch_bytes.argtypes = []
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is ctypes.c_int and name not in ("pot_status_string",):
@@ -241,3 +244,17 @@ def pot_layout_bit(bits: int, kind: int, q: int, b: int) -> tuple[int, int]:
     word, bit = ctypes.c_int(-1), ctypes.c_int(-1)
     _check(lib().pot_layout_bit(bits, kind, q, b, ctypes.byref(word), ctypes.byref(bit)), "pot_layout_bit")
     return word.value, bit.value
+
+
+def pot_gemv_noalloc_max_scratch_bytes() -> int:
+    return int(lib().pot_gemv_noalloc_max_scratch_bytes())
+
+
+def pot_gemv_noalloc(packed_tiled, scales, K: int, bits: int, group: int, x: torch.Tensor, y: torch.Tensor,
+                     stream=None) -> torch.Tensor:
+    """pot_gemv on the tiled layout with the library's built-in scratch array instead of a caller
+    workspace -- for callers that may not allocate device memory.  `y` must be supplied (this wrapper
+    allocates nothing either).  Shapes that need more than pot_gemv_noalloc_max_scratch_bytes() raise."""
+    _check(lib().pot_gemv_noalloc(_ptr(packed_tiled), _ptr(scales), packed_tiled.shape[0], K, bits, group, _ptr(x),
+                                  _ptr(y), _stream(stream)), "pot_gemv_noalloc")
+    return y

@@ -306,3 +306,55 @@ extern "C" pot_status_t uint_gemv(const void* packed, const void* scales, const 
     if (bits == 3) return launch_pdl(gemv_tiled_kernel<3, true>, grid, block, 0, s, P, S, Z, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
     return launch_pdl(gemv_tiled_kernel<4, true>, grid, block, 0, s, P, S, Z, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
 }
+
+// ------------------------------------------------------------------------------------------
+// pot_gemv_noalloc: the split-K GEMV for callers that are not allowed to allocate device memory.
+// ------------------------------------------------------------------------------------------
+// Some hosts of this library own all device memory themselves and hand their plug-ins a fixed
+// budget: an inference server whose serving loop must never hit the implicit device-wide
+// synchronisation of cudaMalloc/cudaFree, or an embedding application whose allocator the
+// library cannot reach.  Such a caller cannot provide the split-K workspace that pot_gemv asks
+// for.  For them the scratch lives in the library image itself: a fixed-size array in device
+// memory that every GPU which loads the library carries until the process exits.
+namespace {
+constexpr size_t kNoAllocScratchBytes = size_t(1) << 20;  // 1 MiB per GPU
+constexpr int kNoAllocMaxDevices = 64;
+}  // namespace
+
+// In host code this name is only a handle for the runtime (it is NOT a device address); the
+// device address is looked up per GPU with cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+namespace {
+std::atomic<void*> g_noalloc_ptr[kNoAllocMaxDevices];
+}
+
+extern "C" size_t pot_gemv_noalloc_max_scratch_bytes(void) { return kNoAllocScratchBytes; }
+
+extern "C" pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales, int64_t N, int64_t K, int bits,
+                                         int group, const void* x, void* y, void* stream) {
+    if (!packed_tiled || !scales || !x || !y) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, bits, group);
+    if (st != POT_OK) return st;
+    if (N % 16 != 0) return POT_ERR_SHAPE;
+    const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
+    if (need > kNoAllocScratchBytes) return POT_ERR_WORKSPACE;  // shape needs more scratch than the built-in array holds
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return POT_ERR_CUDA;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return POT_ERR_UNSUPPORTED;
+    // Set-up, once per device, with that device current: ask the runtime where this GPU's copy of the
+    // array lives.  (Racing first calls both get the same answer, so a plain atomic store is enough.)
+    void* scratch = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return POT_ERR_CUDA;
+        g_noalloc_ptr[dev].store(p, std::memory_order_release);
+        scratch = p;
+    }
+    if (need == 0) return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, nullptr, 0, stream);
+    // The array keeps whatever the previous call left in it.  Only the arrival counters have to start
+    // at zero (the partial sums are fully overwritten before they are read), so clear just those.
+    const size_t counters_bytes = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
+    if (cudaMemsetAsync(scratch, 0, counters_bytes, (cudaStream_t)stream) != cudaSuccess) return POT_ERR_CUDA;
+    return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, need, stream);
+}
