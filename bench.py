@@ -148,7 +148,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config tables (chain only)")
     ap.add_argument("--layers", type=int, default=synth.LLAMA2_7B_LAYERS)
+    ap.add_argument("--kernel", default=None, choices=["gemv", "gemv_uint", "dequant", "dequant_uint", "gemm"],
+                    help="profiling mode: run only this kernel on one small seeded case and print its timing")
+    ap.add_argument("--N", type=int, default=12288)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--M", type=int, default=8)
+    ap.add_argument("--bits", type=int, default=3)
+    ap.add_argument("--no-graph", action="store_true", help="profiling mode: plain stream launches instead of a CUDA graph")
+    ap.add_argument("--copies", type=int, default=16, help="profiling mode: distinct weight copies cycled through (HBM-cold)")
     args = ap.parse_args()
+    if args.kernel:
+        single_kernel(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         reference_arm(args)
@@ -273,6 +284,80 @@ def main():
     del layers3
     if rank == 0:
         print(json.dumps(out))
+
+
+def single_kernel(args):
+    """Profiling mode (used for the ncu captures under profiles/): one kernel, one small case, a few
+    launches over `copies` distinct weight buffers.  Codes are seeded random bytes (every bit pattern is
+    a valid code), scales a seeded spread of legal FP16 values; timing is data-independent."""
+    import torch
+    from paper_2507_11959_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    N, K, bits, M = args.N, args.K, args.bits, args.M
+    g = torch.Generator(device=dev).manual_seed(BASE_PROFILE_SEED)
+    P = [torch.randint(0, 256, (N, K * bits // 8), dtype=torch.uint8, device=dev, generator=g) for _ in range(args.copies)]
+    S = ((torch.rand((N, K // GROUP), device=dev, generator=g) * 0.01 + 0.002).to(torch.float16))
+    Z = torch.randint(0, 1 << bits, (N, K // GROUP), device=dev, generator=g).to(torch.float16)
+    x = torch.randn(K, device=dev, generator=g).to(torch.float16)
+    X = torch.randn((M, K), device=dev, generator=g).to(torch.float16)
+    y = torch.empty(N, dtype=torch.float16, device=dev)
+    Y = torch.empty((M, N), dtype=torch.float16, device=dev)
+    out = torch.empty((N, K), dtype=torch.float16, device=dev) if args.kernel.startswith("dequant") else None
+    ws = B.new_workspace(max(B.pot_gemv_workspace_bytes(N, K, bits, GROUP), B.pot_gemm_workspace_bytes(M, N, K, bits, GROUP)), dev)
+
+    def run(p):
+        st = torch.cuda.current_stream()
+        if args.kernel == "gemv":
+            B.pot_gemv(p, S, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=st)
+        elif args.kernel == "gemv_uint":
+            B.uint_gemv(p, S, Z, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=st)
+        elif args.kernel == "dequant":
+            B.pot_dequant(p, S, K, bits, GROUP, B.F16, out=out, stream=st)
+        elif args.kernel == "dequant_uint":
+            B.uint_dequant(p, S, Z, K, bits, GROUP, B.UINT_FAST, out=out, stream=st)
+        else:
+            B.pot_gemm(p, S, K, bits, GROUP, X, B.TILED, Y=Y, workspace=ws, stream=st)
+
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for p in P[: max(3, args.warmup)]:
+            run(p)
+        stream.synchronize()
+        if args.no_graph:
+            n = 0
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(max(1, args.steps)):
+                for p in P:
+                    run(p)
+                    n += 1
+            e1.record(stream)
+        else:  # one CUDA graph holding one launch per weight copy, replayed `steps` times (no host launch cost)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for p in P:
+                    run(p)
+            g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(max(1, args.steps)):
+                g.replay()
+            e1.record(stream)
+            n = max(1, args.steps) * len(P)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    if args.kernel.startswith("dequant"):
+        nb = N * K * bits // 8 + N * (K // GROUP) * 2 + 2 * N * K
+    else:
+        nb = gemv_bytes(N, K, bits, GROUP, M if args.kernel == "gemm" else 1)
+    print(json.dumps({"kernel": args.kernel, "N": N, "K": K, "M": M, "bits": bits, "graph": not args.no_graph, "us_per_launch": us,
+                      "device_errors": B.pot_debug_errors(),
+                      "GBps": nb / us / 1e3, "launches": n}))
+
+
+BASE_PROFILE_SEED = 250711959
 
 
 def cpu_baseline():

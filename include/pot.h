@@ -89,6 +89,11 @@ size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int g
 
 /* Number of kernels this process has launched through the library (diagnostic counter). */
 uint64_t pot_launch_count(void);
+/* Diagnostics.  Every wait inside the streaming GEMV / small-batch GEMM kernels is bounded; a wait that
+ * gives up records a code in a device word instead of hanging the GPU.  These calls synchronise the
+ * device, return that word (0 = no wait ever gave up) and clear it.                                   */
+int pot_debug_gemv_error(void);
+int pot_debug_gemm_error(void);
 
 /*
  * pot_quantize_ref -- reference PoT quantizer (Eq. 2; groups per Sec. 3.1).  Set-up code: it

@@ -12,160 +12,9 @@
 //  * large M, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
 #include "common.cuh"
 #include "layout.cuh"
+#include "ring.cuh"
 
 namespace pot {
-
-__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                          uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-constexpr int GS_WARPS = 4;
-
-struct GemmSmallPlan {
-    int splits;
-    int chunks_per_split;
-};
-
-inline GemmSmallPlan plan_gemm_small(int64_t N, int64_t K) {
-    const int64_t rbs = N / 16;
-    const int chunks = (int)((K + 511) / 512);
-    int splits = 1;
-    while (rbs * splits < 4 * kSmCount && chunks / (splits * 2) >= GS_WARPS && splits < 16) splits *= 2;
-    GemmSmallPlan p;
-    p.chunks_per_split = (chunks + splits - 1) / splits;
-    p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
-    return p;
-}
-
-// MT = number of 8-token tiles (M <= 8*MT)
-template <int BITS, int MT>
-__global__ void __launch_bounds__(GS_WARPS * 32) pot_gemm_small_kernel(const uint4* __restrict__ packed,
-                                                                        const uint16_t* __restrict__ scales, int64_t N,
-                                                                        int64_t K, int G, int chunks_per_split,
-                                                                        const __half* __restrict__ X, int M,
-                                                                        __half* __restrict__ Y, float* __restrict__ partial,
-                                                                        unsigned* __restrict__ counters) {
-    constexpr int NW = 4 * BITS;
-    __shared__ float red[GS_WARPS][MT][16][8];
-    __shared__ int is_last;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int gid = lane >> 2, tig = lane & 3;
-    const int64_t rb = blockIdx.x;
-    const int split = blockIdx.y, nsplit = gridDim.y;
-    const int64_t ncb = K / 128;
-    const int gpr = (int)(K / G);
-    const int spr = 128 / G;
-    const int chunk_begin = split * chunks_per_split;
-    const int chunk_end = min(chunk_begin + chunks_per_split, (int)((K + 511) / 512));
-
-    float acc[MT][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
-
-    // Lanes whose column block lies beyond K (partial last chunk) keep all-zero records with scale 1.0
-    // and read x as zero: every lane of the warp must still execute the (warp-wide) MMA instructions.
-    uint32_t rec[2][NW];
-    uint32_t sc[2][2];
-    auto load = [&](int chunk) {
-        const int64_t cb = 4 * (int64_t)chunk + tig;
-        if (cb < ncb) {
-            const uint4* unit = packed + (rb * ncb + cb) * (16 * BITS);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                for (int t = 0; t < BITS; ++t) {
-                    const uint4 q = __ldg(unit + t * 16 + gid + 8 * h);
-                    rec[h][4 * t + 0] = q.x; rec[h][4 * t + 1] = q.y; rec[h][4 * t + 2] = q.z; rec[h][4 * t + 3] = q.w;
-                }
-                const uint16_t* sp = scales + (rb * 16 + gid + 8 * h) * gpr + cb * spr;
-                sc[h][0] = (uint32_t)__ldg(sp) * 0x10001u;
-                sc[h][1] = (uint32_t)__ldg(sp + spr - 1) * 0x10001u;
-            }
-        } else {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                for (int i = 0; i < NW; ++i) rec[h][i] = 0u;
-                sc[h][0] = sc[h][1] = 0x3C003C00u;
-            }
-        }
-    };
-    int c = chunk_begin + warp;
-    if (c < chunk_end) load(c);
-    pdl_launch_dependents();
-    pdl_wait();
-    for (; c < chunk_end; c += GS_WARPS) {
-        const int64_t cb = 4 * (int64_t)c + tig;
-        const bool valid = cb < ncb;
-#pragma unroll
-        for (int blk = 0; blk < 8; ++blk) {
-            uint32_t w0[8], w1[8];
-            potl::pot_decode_pairs16<BITS>(rec[0], blk, sc[0][blk >> 2], w0);
-            potl::pot_decode_pairs16<BITS>(rec[1], blk, sc[1][blk >> 2], w1);
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                const int token = 8 * mt + gid;
-                uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
-                if (valid && token < M) {
-                    const uint4* xp = reinterpret_cast<const uint4*>(X + (int64_t)token * K + cb * 128) + 2 * blk;
-                    xa = __ldg(xp);
-                    xb = __ldg(xp + 1);
-                }
-                mma_16816(acc[mt], w0[0], w1[0], w0[1], w1[1], xa.x, xa.y);
-                mma_16816(acc[mt], w0[2], w1[2], w0[3], w1[3], xa.z, xa.w);
-                mma_16816(acc[mt], w0[4], w1[4], w0[5], w1[5], xb.x, xb.y);
-                mma_16816(acc[mt], w0[6], w1[6], w0[7], w1[7], xb.z, xb.w);
-            }
-        }
-        if (c + GS_WARPS < chunk_end) load(c + GS_WARPS);
-    }
-    // accumulator (row gid / gid+8, token 2tig / 2tig+1) -> shared, then sum the warps
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        red[warp][mt][gid][2 * tig] = acc[mt][0];
-        red[warp][mt][gid][2 * tig + 1] = acc[mt][1];
-        red[warp][mt][gid + 8][2 * tig] = acc[mt][2];
-        red[warp][mt][gid + 8][2 * tig + 1] = acc[mt][3];
-    }
-    __syncthreads();
-    // thread -> (token, row): consecutive threads take consecutive rows, so stores to Y[token][rows] coalesce
-    for (int e = threadIdx.x; e < MT * 8 * 16; e += GS_WARPS * 32) {
-        const int r = e & 15, token = e >> 4;
-        if (token >= M) continue;
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < GS_WARPS; ++w) s += red[w][token >> 3][r][token & 7];
-        const int64_t row = rb * 16 + r;
-        if (nsplit == 1) Y[(int64_t)token * N + row] = __float2half_rn(s);
-        else partial[((int64_t)split * M + token) * N + row] = s;
-    }
-    if (nsplit == 1) return;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned prev = atomicAdd(&counters[rb], 1u);
-        is_last = (prev == (unsigned)nsplit - 1u);
-        if (is_last) counters[rb] = 0u;
-    }
-    __syncthreads();
-    if (is_last) {
-        __threadfence();
-        for (int e = threadIdx.x; e < MT * 8 * 16; e += GS_WARPS * 32) {
-            const int r = e & 15, token = e >> 4;
-            if (token >= M) continue;
-            const int64_t row = rb * 16 + r;
-            float s = 0.f;
-            for (int sp = 0; sp < nsplit; ++sp) s += __ldcg(partial + ((int64_t)sp * M + token) * N + row);
-            Y[(int64_t)token * N + row] = __float2half_rn(s);
-        }
-    }
-}
 
 // ------------------------------------------------------------------------------------------
 // fallback: canonical layout, any M.  64 tokens x 64 rows x 128 columns per CTA step.
@@ -241,7 +90,7 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
 #pragma unroll
             for (int i = 0; i < 2; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) mma_16816(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
+                for (int j = 0; j < 4; ++j) rg_mma(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
         }
     }
 #pragma unroll
@@ -272,14 +121,11 @@ static bool use_small(int64_t M, int64_t N, pot_layout_t layout) {
     return layout == POT_LAYOUT_TILED && M <= 32 && N % 16 == 0;
 }
 
+static int small_mt(int64_t M) { return M <= 8 ? 1 : (M <= 16 ? 2 : 4); }
+
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || M <= 0) return 0;
-    if (M <= 32 && N % 16 == 0) {
-        const GemmSmallPlan p = plan_gemm_small(N, K);
-        if (p.splits == 1) return 0;
-        const size_t counters = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
-        return counters + (size_t)p.splits * (size_t)M * (size_t)N * 4;
-    }
+    if (M <= 32 && N % 16 == 0) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
@@ -296,19 +142,10 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
         return POT_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;
     if (use_small(M, N, layout)) {
-        const GemmSmallPlan p = plan_gemm_small(N, K);
         const size_t need = pot_gemm_workspace_bytes(M, N, K, bits, group);
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-        const size_t counters_bytes = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
-        unsigned* counters = (unsigned*)workspace;
-        float* partial = need ? (float*)((char*)workspace + counters_bytes) : nullptr;
-        const dim3 grid((unsigned)(N / 16), (unsigned)p.splits), block(GS_WARPS * 32);
-        auto* P = (const uint4*)packed;
-        auto* S = (const uint16_t*)scales;
-        auto* Xp = (const __half*)X;
-        auto* Yp = (__half*)Y;
         const int Mi = (int)M;
-#define POT_GS(B, T) return launch_pdl(pot_gemm_small_kernel<B, T>, grid, block, 0, s, P, S, N, K, group, p.chunks_per_split, Xp, Mi, Yp, partial, counters)
+#define POT_GS(B, T) return launch_ring<B, RG_POT_MMA, T>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, ring_error_ptr(), s)
 #define POT_GS_B(B)                  \
     if (M <= 8) POT_GS(B, 1);        \
     else if (M <= 16) POT_GS(B, 2);  \
@@ -328,3 +165,8 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
     if (bits == 3) return launch_pdl(pot_gemm_fallback_kernel<3>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (__half*)Y);
     return launch_pdl(pot_gemm_fallback_kernel<4>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (__half*)Y);
 }
+
+// Diagnostic: reads and clears the device error word of the gemm kernels in this library (0 = every bounded
+// wait completed; 1 = a producer gave up waiting for a free ring slot; 2 = a consumer gave up waiting for
+// data).  Synchronises the device.
+extern "C" int pot_debug_gemm_error(void) { return ring_error_fetch(); }

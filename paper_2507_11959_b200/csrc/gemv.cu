@@ -4,11 +4,10 @@
 // (fma.rn.f32.f16: FP16 operands, FP32 accumulator), K is reduced across lanes with warp
 // shuffles and, when N alone cannot fill 148 SMs, split across CTAs.
 //
-//  * tiled layout (the fast path): one warp-step covers 16 rows x 512 columns.  Lane
-//    (gid = lane/4, tig = lane%4) owns the 128-code records of rows gid and gid+8 in column
-//    block 4*chunk + tig, i.e. exactly one quantization group per record (two for G = 64), so
-//    the scale pattern added to every pair is a loop constant.  The 16-byte loads of a warp
-//    cover whole 128-byte lines.
+//  * tiled layout (the fast path): the ring-buffered streaming kernel of ring.cuh.  One warp-step covers
+//    16 rows x 512 columns; a lane owns the 128-code records of two rows in one column block,
+//    i.e. exactly one quantization group per record (two for G = 64), so the scale pattern added
+//    to every pair is a loop constant.  The 16-byte loads of a warp cover whole 128-byte lines.
 //  * canonical layout (any N): one warp per row, 8 codes per lane per step.
 //
 // Programmatic dependent launch: weights and scales do not depend on the previous kernel in
@@ -17,21 +16,9 @@
 // ramp-up of one GEMV overlaps the tail of the previous one.
 #include "common.cuh"
 #include "layout.cuh"
+#include "ring.cuh"
 
 namespace pot {
-
-// acc += w.lo * x.lo + w.hi * x.hi, FP16 operands, FP32 accumulation, one rounding per FMA.
-__device__ __forceinline__ void fma2_f32_f16(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
-    asm("{\n\t"
-        ".reg .b16 wl, wh, xl, xh;\n\t"
-        "mov.b32 {wl, wh}, %2;\n\t"
-        "mov.b32 {xl, xh}, %3;\n\t"
-        "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
-        "fma.rn.f32.f16 %1, wh, xh, %1;\n\t"
-        "}"
-        : "+f"(acc0), "+f"(acc1)
-        : "r"(w2), "r"(x2));
-}
 
 // ------------------------------------------------------------------------------------------
 // canonical layout, one warp per row
@@ -72,144 +59,12 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
                 const __half2 w = __hmul2(d, __half2half2(__ushort_as_half((uint16_t)s16)));
                 w2 = *reinterpret_cast<const uint32_t*>(&w);
             }
-            fma2_f32_f16(acc0, acc1, w2, xs[j]);
+            rg_fma2(acc0, acc1, w2, xs[j]);
         }
     }
     float acc = acc0 + acc1;
     for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) y[row] = __float2half_rn(acc);
-}
-
-// ------------------------------------------------------------------------------------------
-// tiled layout, PoT
-// ------------------------------------------------------------------------------------------
-constexpr int GV_WARPS = 4;
-
-struct GemvPlan {
-    int splits;            // CTAs along K per 16-row block
-    int chunks_per_split;  // 512-column chunks per CTA
-};
-
-inline GemvPlan plan_gemv(int64_t N, int64_t K) {
-    const int64_t rbs = N / 16;
-    const int chunks = (int)((K + 511) / 512);
-    // aim for at least ~4 CTAs per SM while every warp of a CTA keeps at least one chunk
-    int splits = 1;
-    while (rbs * splits < 4 * kSmCount && chunks / (splits * 2) >= GV_WARPS && splits < 16) splits *= 2;
-    GemvPlan p;
-    p.chunks_per_split = (chunks + splits - 1) / splits;
-    p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
-    return p;
-}
-
-template <int BITS, bool UNIFORM>
-__global__ void __launch_bounds__(GV_WARPS * 32) gemv_tiled_kernel(const uint4* __restrict__ packed,
-                                                                    const uint16_t* __restrict__ scales,
-                                                                    const uint16_t* __restrict__ zeros, int64_t N,
-                                                                    int64_t K, int G, int chunks_per_split,
-                                                                        const uint4* __restrict__ x,
-                                                                        __half* __restrict__ y, float* __restrict__ partial,
-                                                                        unsigned* __restrict__ counters) {
-    constexpr int NW = 4 * BITS;  // 32-bit words per record
-    __shared__ float red[GV_WARPS][16];
-    __shared__ int is_last;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int gid = lane >> 2, tig = lane & 3;
-    const int64_t rb = blockIdx.x;
-    const int split = blockIdx.y, nsplit = gridDim.y;
-    const int64_t ncb = K / 128;
-    const int gpr = (int)(K / G);          // groups per row
-    const int spr = 128 / G;               // scales per record (1 or 2)
-    const int chunk_begin = split * chunks_per_split;
-    const int chunk_end = min(chunk_begin + chunks_per_split, (int)((K + 511) / 512));
-
-    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-    uint32_t rec[2][NW];
-    uint32_t sc[2][2];
-    uint32_t zp[2][2];  // uniform twin only: zero-points
-    int c = chunk_begin + warp;
-    auto load = [&](int chunk) {
-        const int64_t cb = 4 * (int64_t)chunk + tig;
-        if (cb < ncb) {
-            const uint4* unit = packed + (rb * ncb + cb) * (16 * BITS);  // 16 rows x BITS 16-byte words
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                for (int t = 0; t < BITS; ++t) {
-                    const uint4 q = __ldg(unit + t * 16 + gid + 8 * h);
-                    rec[h][4 * t + 0] = q.x; rec[h][4 * t + 1] = q.y; rec[h][4 * t + 2] = q.z; rec[h][4 * t + 3] = q.w;
-                }
-                const uint16_t* sp = scales + (rb * 16 + gid + 8 * h) * gpr + cb * spr;
-                sc[h][0] = (uint32_t)__ldg(sp) * 0x10001u;
-                sc[h][1] = (uint32_t)__ldg(sp + spr - 1) * 0x10001u;
-                if constexpr (UNIFORM) {
-                    const uint16_t* zq = zeros + (rb * 16 + gid + 8 * h) * gpr + cb * spr;
-                    zp[h][0] = (uint32_t)__ldg(zq) * 0x10001u;
-                    zp[h][1] = (uint32_t)__ldg(zq + spr - 1) * 0x10001u;
-                }
-            }
-        }
-    };
-    if (c < chunk_end) load(c);
-    pdl_launch_dependents();
-    pdl_wait();  // x (and the buffers written below) may belong to the previous kernel in the stream
-    for (; c < chunk_end; c += GV_WARPS) {
-        const int64_t cb = 4 * (int64_t)c + tig;
-        if (cb < ncb) {
-            const uint4* xp = x + cb * 16;  // 128 halves = 16 x 16 bytes
-#pragma unroll
-            for (int blk = 0; blk < 8; ++blk) {
-                const uint4 xa = __ldg(xp + 2 * blk), xb = __ldg(xp + 2 * blk + 1);
-                const uint32_t xs[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t w2[8];
-                    if constexpr (!UNIFORM) {
-                        potl::pot_decode_pairs16<BITS>(rec[h], blk, sc[h][blk >> 2], w2);
-                    } else {
-                        potl::UintParams pr;
-                        pr.s2 = potl::bits_h2(sc[h][blk >> 2]);
-                        pr.z = potl::bits_h2(zp[h][blk >> 2]);
-                        potl::uint_decode_pairs16<BITS>(rec[h], blk, pr, w2);
-                    }
-#pragma unroll
-                    for (int p = 0; p < 8; ++p) fma2_f32_f16(acc[h][0], acc[h][1], w2[p], xs[p]);
-                }
-            }
-        }
-        if (c + GV_WARPS < chunk_end) load(c + GV_WARPS);
-    }
-    // K-reduction: across the 4 lanes that share a row, then across warps
-    float r0 = acc[0][0] + acc[0][1], r1 = acc[1][0] + acc[1][1];
-    r0 += __shfl_xor_sync(0xffffffffu, r0, 1); r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
-    r1 += __shfl_xor_sync(0xffffffffu, r1, 1); r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
-    if (tig == 0) { red[warp][gid] = r0; red[warp][gid + 8] = r1; }
-    __syncthreads();
-    if (threadIdx.x < 16) {
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < GV_WARPS; ++w) s += red[w][threadIdx.x];
-        const int64_t row = rb * 16 + threadIdx.x;
-        if (nsplit == 1) y[row] = __float2half_rn(s);
-        else partial[(int64_t)split * N + row] = s;
-    }
-    if (nsplit == 1) return;
-    // split-K: the CTA that arrives last for this row block sums the partials in split order
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned prev = atomicAdd(&counters[rb], 1u);
-        is_last = (prev == (unsigned)nsplit - 1u);
-        if (is_last) counters[rb] = 0u;  // leave the workspace ready for the next call
-    }
-    __syncthreads();
-    if (is_last && threadIdx.x < 16) {
-        __threadfence();
-        const int64_t row = rb * 16 + threadIdx.x;
-        float s = 0.f;
-        for (int sp = 0; sp < nsplit; ++sp) s += __ldcg(partial + (int64_t)sp * N + row);
-        y[row] = __float2half_rn(s);
-    }
 }
 
 }  // namespace pot
@@ -218,11 +73,7 @@ using namespace pot;
 
 extern "C" size_t pot_gemv_workspace_bytes(int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || N % 16 != 0) return 0;
-    const GemvPlan p = plan_gemv(N, K);
-    if (p.splits == 1) return 0;
-    // counters (one per 16-row block, padded to 256 bytes) + FP32 partials [splits][N]
-    const size_t counters = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
-    return counters + (size_t)p.splits * (size_t)N * 4;
+    return plan_ring(N, K, 1, bits, 1).ws_bytes;  // row-block step counters + FP32 partial slots
 }
 
 extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -244,19 +95,11 @@ extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t
         return launch_pdl(gemv_canonical_kernel<4, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
     }
     if (N % 16 != 0) return POT_ERR_SHAPE;
-    const GemvPlan p = plan_gemv(N, K);
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
     if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-    const size_t counters_bytes = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
-    unsigned* counters = (unsigned*)workspace;
-    float* partial = need ? (float*)((char*)workspace + counters_bytes) : nullptr;
-    const dim3 grid((unsigned)(N / 16), (unsigned)p.splits), block(GV_WARPS * 32);
-    auto* P = (const uint4*)packed;
-    auto* S = (const uint16_t*)scales;
-    const uint16_t* Zn = nullptr;
-    if (bits == 2) return launch_pdl(gemv_tiled_kernel<2, false>, grid, block, 0, s, P, S, Zn, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
-    if (bits == 3) return launch_pdl(gemv_tiled_kernel<3, false>, grid, block, 0, s, P, S, Zn, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
-    return launch_pdl(gemv_tiled_kernel<4, false>, grid, block, 0, s, P, S, Zn, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
+    if (bits == 2) return launch_ring<2, RG_POT_FMA, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
+    if (bits == 3) return launch_ring<3, RG_POT_FMA, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
+    return launch_ring<4, RG_POT_FMA, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
 }
 
 extern "C" pot_status_t pot_gemv_host(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -294,17 +137,11 @@ extern "C" pot_status_t uint_gemv(const void* packed, const void* scales, const 
         return launch_pdl(gemv_canonical_kernel<4, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (__half*)y);
     }
     if (N % 16 != 0) return POT_ERR_SHAPE;
-    const GemvPlan p = plan_gemv(N, K);
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
     if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-    const size_t counters_bytes = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
-    unsigned* counters = (unsigned*)workspace;
-    float* partial = need ? (float*)((char*)workspace + counters_bytes) : nullptr;
-    const dim3 grid((unsigned)(N / 16), (unsigned)p.splits), block(GV_WARPS * 32);
-    auto* P = (const uint4*)packed;
-    if (bits == 2) return launch_pdl(gemv_tiled_kernel<2, true>, grid, block, 0, s, P, S, Z, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
-    if (bits == 3) return launch_pdl(gemv_tiled_kernel<3, true>, grid, block, 0, s, P, S, Z, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
-    return launch_pdl(gemv_tiled_kernel<4, true>, grid, block, 0, s, P, S, Z, N, K, group, p.chunks_per_split, (const uint4*)x, (__half*)y, partial, counters);
+    if (bits == 2) return launch_ring<2, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
+    if (bits == 3) return launch_ring<3, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
+    return launch_ring<4, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -354,7 +191,12 @@ extern "C" pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* s
     if (need == 0) return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, nullptr, 0, stream);
     // The array keeps whatever the previous call left in it.  Only the arrival counters have to start
     // at zero (the partial sums are fully overwritten before they are read), so clear just those.
-    const size_t counters_bytes = ((size_t)(N / 16) * 4 + 255) / 256 * 256;
+    const size_t counters_bytes = plan_ring(N, K, 1, bits, 1).ws_counters;
     if (cudaMemsetAsync(scratch, 0, counters_bytes, (cudaStream_t)stream) != cudaSuccess) return POT_ERR_CUDA;
     return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, need, stream);
 }
+
+// Diagnostic: reads and clears the device error word of the gemv kernels in this library (0 = every bounded
+// wait completed; 1 = a producer gave up waiting for a free ring slot; 2 = a consumer gave up waiting for
+// data).  Synchronises the device.
+extern "C" int pot_debug_gemv_error(void) { return ring_error_fetch(); }

@@ -13,8 +13,16 @@
 //                p <= 5 : anchor 2p + 16h           (decoded straight from the word)
 //                p == 6 : anchor 28 (h=0), 12 (h=1) (decoded after rotating the word left by 8)
 //                p == 7 : anchor 30 (h=0), 14 (h=1)
-//  PoT n = 3 : words 0..7 hold the 2-bit exponents, word w = q/16, bits 2p + 16h + {0,1};
-//              words 8..11 hold the signs, word 8 + q/32, bit (q%32)/2 + 16h.
+//  PoT n = 3 : the record is four "triples" of three words; triple T = q/32 holds pairs
+//              P = (q%32)/2 = 0..15.  Pair P < 15 lives in word 3T + P/5 as slot d = P%5:
+//                d < 4 : exponent at bits 3d, 3d+1 and sign at 3d+5 (+16h) -- the sign sits five
+//                        positions above the exponent's low bit, so ONE mask and ONE shift-add
+//                        place both (these are 12 of every 16 pairs);
+//                d = 4 : exponent at bits 12,13 and sign already at bit 15 (+16h);
+//              pair 15 is spread over bit 2 (+16h) of the three words: exponent bit 0 in word
+//              3T, exponent bit 1 in word 3T+1, sign in word 3T+2.
+//              (The uniform twin keeps the plain plane map: words 0..7 hold the low two bits as
+//              fields 2p + 16h, words 8..11 the high bit at (q%32)/2 + 16h.)
 //  PoT n = 4 : word w = q/8 holds codes 8w..8w+7; pair p = (q%8)/2; exponent at bits
 //              3p + 16h + {0,1,2}, sign at bit 12 + p + 16h.
 //  uniform   : the n-bit integer code as a field: n = 2 at 2p + 16h (p < 8), n = 4 at
@@ -47,13 +55,24 @@ __host__ __device__ inline BitPos record_bit(int bits, int kind, int q, int b) {
             else anchor = h ? 14 : 30;
             r.bit = (b == 0) ? anchor : ((anchor + 5) & 31);
         }
-    } else if (bits == 3) {
+    } else if (bits == 3 && kind == KIND_UINT) {
         if (b < 2) {
             r.word = q >> 4;
             r.bit = 2 * ((q & 15) >> 1) + 16 * h + b;
         } else {
             r.word = 8 + (q >> 5);
             r.bit = ((q & 31) >> 1) + 16 * h;
+        }
+    } else if (bits == 3) {
+        const int T = q >> 5, P = (q & 31) >> 1;
+        if (P < 15) {
+            const int d = P % 5;
+            r.word = 3 * T + P / 5;
+            if (d < 4) r.bit = 3 * d + 16 * h + (b < 2 ? b : 5);
+            else r.bit = 16 * h + (b < 2 ? 12 + b : 15);
+        } else {
+            r.word = 3 * T + b;
+            r.bit = 2 + 16 * h;
         }
     } else {
         r.word = q >> 3;
@@ -108,49 +127,55 @@ struct PotDecoder<4> {
     }
 };
 
-// n = 3 : exponent plane word (8 pairs) + the matching half of a sign-plane word.
+// n = 3 : three words hold 16 pairs (see the map at the top of this file).
 template <>
 struct PotDecoder<3> {
     static constexpr int WORDS = 12;
-    static constexpr int PAIRS_PER_WORD = 8;
-    // we: exponent word j (0..7); ws: sign word 8 + j/2; `upper` = j & 1 selects sign bits 8..15
-    static __device__ __forceinline__ void word(uint32_t we, uint32_t ws, int upper, uint32_t sc2,
-                                                uint32_t (&out)[8]) {
-        const uint32_t r = rotl(we, 24);  // brings fields 6,7 (bits 12..15) down to bits 4..7
+    // out[16]: pairs 16T .. 16T+15 of the record, from words w0, w1, w2 of triple T
+    static __device__ __forceinline__ void triple(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sc2,
+                                                  uint32_t (&out)[16]) {
+        const uint32_t w[3] = {w0, w1, w2};
 #pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            uint32_t e;
-            if (p < 6) e = mad(we & (0x00030003u << (2 * p)), 1u << (10 - 2 * p), sc2);
-            else e = mad(r & (0x00030003u << (2 * p - 8)), 1u << (18 - 2 * p), sc2);
-            const int sp = p + 8 * upper;  // sign bit position inside each half of ws
-            if (sp == 15) out[p] = e | (ws & 0x80008000u);
-            else out[p] = mad(ws & (0x00010001u << sp), 1u << (15 - sp), e);
+        for (int j = 0; j < 3; ++j) {
+#pragma unroll
+            for (int d = 0; d < 4; ++d) out[5 * j + d] = mad(w[j] & (0x00230023u << (3 * d)), 1u << (10 - 3 * d), sc2);
+            // slot 4: exponent at bits 12,13 (two positions too high), sign in place at bit 15
+            const uint32_t e = (__funnelshift_r(w[j], w[j], 2) & 0x0C000C00u) + sc2;
+            out[5 * j + 4] = e | (w[j] & 0x80008000u);
         }
+        uint32_t y = mad(w0 & 0x00040004u, 1u << 8, sc2);
+        y = mad(w1 & 0x00040004u, 1u << 9, y);
+        out[15] = mad(w2 & 0x00040004u, 1u << 13, y);
     }
 };
 
-// Decode a whole record (4n words in registers) into 64 half2 patterns, pair order 0..63.
+// Decode 32 consecutive codes (16 pairs): quarter T (0..3) of a record held in registers.
 template <int BITS>
-__device__ __forceinline__ void pot_decode_pairs16(const uint32_t* rec, int blk, uint32_t sc2, uint32_t (&out)[8]);
+__device__ __forceinline__ void pot_decode32(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]);
 
-// blk = index of a 16-code block (8 pairs) inside the record, 0..7
 template <>
-__device__ __forceinline__ void pot_decode_pairs16<2>(const uint32_t* rec, int blk, uint32_t sc2, uint32_t (&out)[8]) {
-    PotDecoder<2>::word(rec[blk], sc2, out);
+__device__ __forceinline__ void pot_decode32<2>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
+    uint32_t a[8], b[8];
+    PotDecoder<2>::word(rec[2 * T], sc2, a);
+    PotDecoder<2>::word(rec[2 * T + 1], sc2, b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        out[i] = a[i];
+        out[8 + i] = b[i];
+    }
 }
 template <>
-__device__ __forceinline__ void pot_decode_pairs16<3>(const uint32_t* rec, int blk, uint32_t sc2, uint32_t (&out)[8]) {
-    PotDecoder<3>::word(rec[blk], rec[8 + (blk >> 1)], blk & 1, sc2, out);
+__device__ __forceinline__ void pot_decode32<3>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
+    PotDecoder<3>::triple(rec[3 * T], rec[3 * T + 1], rec[3 * T + 2], sc2, out);
 }
 template <>
-__device__ __forceinline__ void pot_decode_pairs16<4>(const uint32_t* rec, int blk, uint32_t sc2, uint32_t (&out)[8]) {
-    uint32_t a[4], b[4];
-    PotDecoder<4>::word(rec[2 * blk], sc2, a);
-    PotDecoder<4>::word(rec[2 * blk + 1], sc2, b);
+__device__ __forceinline__ void pot_decode32<4>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        out[i] = a[i];
-        out[4 + i] = b[i];
+        uint32_t a[4];
+        PotDecoder<4>::word(rec[4 * T + i], sc2, a);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) out[4 * i + k] = a[k];
     }
 }
 
@@ -222,6 +247,18 @@ __device__ __forceinline__ void uint_decode_pairs16<3>(const uint32_t* rec, int 
         const uint32_t hb = (ws >> p) & 0x00010001u;
         const uint32_t h = hb * 4u + lo;  // 1024 + q
         out[p] = h2_bits(__hmul2(__hsub2(bits_h2(h), zm), pr.s2));
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void uint_decode32(const uint32_t* rec, int T, const UintParams& pr, uint32_t (&out)[16]) {
+    uint32_t a[8], b[8];
+    uint_decode_pairs16<BITS>(rec, 2 * T, pr, a);
+    uint_decode_pairs16<BITS>(rec, 2 * T + 1, pr, b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        out[i] = a[i];
+        out[8 + i] = b[i];
     }
 }
 #endif  // __CUDACC__

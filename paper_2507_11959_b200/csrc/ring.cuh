@@ -1,0 +1,472 @@
+// Ring-buffered streaming kernel for the decode GEMV (CUDA cores) and the small-batch GEMM (tensor
+// cores) on the tiled layout.
+//
+// One persistent CTA per SM.  A producer warp streams the CTA's share of the packed codes from
+// HBM into a shared-memory ring with 1-D bulk copies (cp.async.bulk + mbarrier transaction
+// counts), several steps (up to 20 KB) per copy since the share is one contiguous byte range in the
+// tiled layout; the bytes in flight therefore cost no registers, and the whole share of a short
+// matrix can be requested before the first byte arrives.  Consumer warps take the ring stages
+// round-robin, pull their records out of shared memory with conflict-free 16-byte loads, decode
+// them in registers (integer mask / shift-add into the scale's bit pattern) and accumulate in
+// FP32 -- with the mixed-precision FMA (GEMV) or with warp-level MMAs whose A fragment is the
+// decoded weights (small batch).
+//
+// Work decomposition: the matrix is a sequence of steps; step g = 16 rows x 512 columns
+// (row block g / spr, columns 512 * (g % spr)).  CTA b owns the contiguous range
+// [b*G/grid, (b+1)*G/grid), so every SM streams the same number of bytes (+-1 step).  Each step
+// yields 16 (x tokens) FP32 partial sums; when a row block needs more than one step they go to a
+// slot of the workspace indexed by (row block, step) and the warp that delivers the last slot
+// of a row block (a per-row-block counter tells it) adds the slots in ascending column order --
+// the result is independent of timing.  No warp ever waits for another CTA.
+//
+// Every mbarrier wait is bounded: after kSpinLimit polls the waiter records an error code in
+// *err (when given), and carries on without the data, so a lost copy cannot hang the GPU.
+#pragma once
+#include "common.cuh"
+#include "layout.cuh"
+
+namespace pot {
+
+constexpr int RG_CONSUMERS = 15;
+constexpr int RG_THREADS = (RG_CONSUMERS + 1) * 32;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2 };
+
+constexpr int RG_Q = 5;  // steps per ring slot (one bulk copy) = warps per consumer group
+constexpr int RG_GROUPS = RG_CONSUMERS / RG_Q;  // slot m is consumed by group m % RG_GROUPS, warp i of it takes step i
+static_assert(RG_GROUPS * RG_Q == RG_CONSUMERS, "consumer warps must split into whole groups");
+__host__ __device__ constexpr int rg_unit_bytes(int bits) { return 256 * bits; }
+__host__ __device__ constexpr int rg_slot_bytes(int bits) { return RG_Q * 4 * rg_unit_bytes(bits); }
+
+struct RingPlan {
+    int grid;
+    int spr;
+    int64_t total_steps;
+    int stages;
+    bool x_in_smem;
+    size_t x_bytes;      // shared-memory bytes for the staged activations (0 if read from global)
+    size_t cmb_bytes;    // shared-memory bytes for combining the steps of a row block inside the CTA (0 = off)
+    size_t smem_bytes;   // total dynamic shared memory
+    size_t ws_counters;
+    size_t ws_bytes;
+};
+
+inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok) {
+    RingPlan p;
+    const int64_t nrb = N / 16, ncb = K / 128;
+    p.spr = (int)((ncb + 3) / 4);
+    p.total_steps = nrb * p.spr;
+    p.grid = (int)(p.total_steps < kSmCount ? p.total_steps : kSmCount);
+    const size_t xb = (size_t)M * (size_t)K * 2;
+    p.x_in_smem = xb <= 64 * 1024;
+    p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
+    const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
+    // per step one slot of 16*tok floats, plus one counter per local row block
+    p.cmb_bytes = (size_t)(per_cta + 1) * 64 * (size_t)tok + (size_t)(per_cta / p.spr + 3) * 4;
+    p.cmb_bytes = (p.cmb_bytes + 127) / 128 * 128;
+    if (p.spr == 1 || p.cmb_bytes > 48 * 1024) p.cmb_bytes = 0;
+    const size_t budget = 200 * 1024 - p.x_bytes - p.cmb_bytes - 1024;  // room for barriers and the runtime's reserve
+    int64_t st = (int64_t)(budget / (size_t)rg_slot_bytes(bits));
+    const int64_t slots_needed = (per_cta + RG_Q - 1) / RG_Q;
+    if (st > 63) st = 63;
+    // A slot that is reused must always come back to the same group of consumer warps (see the kernel):
+    // the ring length is a multiple of the number of groups unless it holds the CTA's whole share.
+    if (st >= slots_needed) st = slots_needed;
+    else st = st / RG_GROUPS * RG_GROUPS;
+    if (st < 1) st = 1;
+    p.stages = (int)st;
+    p.smem_bytes = 1024 + p.x_bytes + p.cmb_bytes + (size_t)p.stages * (size_t)rg_slot_bytes(bits);
+    p.ws_counters = ((size_t)nrb * 4 + 255) / 256 * 256;
+    p.ws_bytes = p.spr > 1 ? p.ws_counters + (size_t)nrb * (size_t)p.spr * 16 * (size_t)tok * 4 : 0;
+    return p;
+}
+
+// ---- mbarrier / bulk-copy primitives ---------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// bounded wait: false after kSpinLimit unsuccessful polls
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(RG_CONSUMERS * 32) : "memory"); }
+
+__device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
+    asm("{\n\t"
+        ".reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %2;\n\t"
+        "mov.b32 {xl, xh}, %3;\n\t"
+        "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
+        "fma.rn.f32.f16 %1, wh, xh, %1;\n\t"
+        "}"
+        : "+f"(acc0), "+f"(acc1)
+        : "r"(w2), "r"(x2));
+}
+__device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// MODE RG_POT_FMA / RG_UINT_FMA: M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
+template <int BITS, int MODE, int MT, bool XSMEM>
+__global__ void __launch_bounds__(RG_THREADS, 1)
+ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
+            int64_t N, int64_t K, int G, int spr, int64_t total_steps, int stages, int x_bytes, int cmb_bytes,
+            const __half* __restrict__ X, int M, __half* __restrict__ Y, float* __restrict__ partial,
+            unsigned* __restrict__ counters, int* __restrict__ err) {
+    constexpr int NW = 4 * BITS;
+    constexpr bool MMA = (MODE == RG_POT_MMA);
+    constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
+    constexpr int TOK = MMA ? 8 * MT : 1;
+    constexpr int SLOT = rg_slot_bytes(BITS);
+    constexpr int UB = rg_unit_bytes(BITS);
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);  // full[stages], empty[stages]  (<= 1024 bytes)
+    const uint4* xs = reinterpret_cast<const uint4*>(smem + 1024);
+    float* cmb = reinterpret_cast<float*>(smem + 1024 + x_bytes);  // [nsteps][16*TOK] partial slots, then counters
+    unsigned char* ring = smem + 1024 + x_bytes + cmb_bytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t ncb = K / 128;
+    const int64_t g_begin = (int64_t)blockIdx.x * total_steps / gridDim.x;
+    const int64_t g_end = ((int64_t)blockIdx.x + 1) * total_steps / gridDim.x;
+    const int nsteps = (int)(g_end - g_begin);
+    const int nmacro = (nsteps + RG_Q - 1) / RG_Q;
+    // global unit index (16 rows x 128 columns each, stored contiguously) at which step g starts
+    auto unit_index = [&](int64_t g) -> int64_t {  // the step count fits 32 bits: cheap division
+        const uint32_t rbq = (uint32_t)g / (uint32_t)spr;
+        return (int64_t)rbq * ncb + 4 * (int64_t)((uint32_t)g - rbq * (uint32_t)spr);
+    };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&bars[s]), 1);                // full: the producer's expect_tx arrival
+            mbar_init(smem_u32(&bars[stages + s]), RG_Q);    // empty: one arrival per consumed step
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    unsigned* cmb_cnt = reinterpret_cast<unsigned*>(cmb + (size_t)(nsteps + 1) * 16 * TOK);
+    if (cmb_bytes) {
+        for (int i = threadIdx.x; i < nsteps / spr + 3; i += blockDim.x) cmb_cnt[i] = 0u;
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == RG_CONSUMERS) {
+        // ---------------- producer: weights do not depend on the previous kernel, start at once ----------
+        if (lane == 0) {
+            for (int m = 0; m < nmacro; ++m) {
+                const int slot = m % stages;
+                if (m >= stages) {
+                    if (!mbar_wait(smem_u32(&bars[stages + slot]), (uint32_t)((m / stages - 1) & 1))) {
+                        if (err) atomicCAS(err, 0, 1 | (m << 8) | (nsteps << 16));  // first failure wins
+                    }
+                }
+                const int64_t gs = g_begin + (int64_t)m * RG_Q;
+                const int64_t ge = gs + RG_Q < g_end ? gs + RG_Q : g_end;
+                const int64_t u0 = unit_index(gs);
+                const uint32_t bytes = (uint32_t)((unit_index(ge) - u0) * UB);
+                const uint32_t full = smem_u32(&bars[slot]);
+                mbar_expect_tx(full, bytes);
+                bulk_g2s(smem_u32(ring + (size_t)slot * SLOT), packed + u0 * (16 * BITS), bytes, full);
+            }
+        }
+        return;
+    }
+
+    // -------------------- consumers --------------------------------------------------------------------
+    const int gid = MMA ? (lane >> 2) : (lane & 7);
+    const int tig = MMA ? (lane & 3) : (lane >> 3);
+    const int gpr = (int)(K / G);
+    const int spg = 128 / G;
+
+    // scales (and zero-points) of a step are fetched one step ahead, straight from global memory
+    uint32_t sc[2][2][2], zp[2][2][2];
+    auto load_scales = [&](int64_t rb, int c, int buf) {
+        const int64_t cb = 4 * (int64_t)c + tig;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            sc[buf][h][0] = sc[buf][h][1] = 0x3C003C00u;
+            zp[buf][h][0] = zp[buf][h][1] = 0u;
+            if (cb < ncb) {
+                const int64_t so = (rb * 16 + gid + 8 * h) * gpr + cb * spg;
+                sc[buf][h][0] = (uint32_t)__ldg(scales + so) * 0x10001u;
+                sc[buf][h][1] = (uint32_t)__ldg(scales + so + spg - 1) * 0x10001u;
+                if constexpr (UNIFORM) {
+                    zp[buf][h][0] = (uint32_t)__ldg(zeros + so) * 0x10001u;
+                    zp[buf][h][1] = (uint32_t)__ldg(zeros + so + spg - 1) * 0x10001u;
+                }
+            }
+        }
+    };
+    // Slot (bulk copy) m holds steps m*Q .. m*Q+Q-1 and belongs to warp group m % GROUPS; warp i of the group
+    // takes step m*Q + i.  A warp therefore meets the barriers of "its" slots once per fill and in order,
+    // which is what the one-bit phase parity of an mbarrier requires.
+    const int grp = warp / RG_Q, wig = warp - grp * RG_Q;
+    const int j_first = grp * RG_Q + wig;             // this warp's first step (local index)
+    constexpr int J_STRIDE = RG_GROUPS * RG_Q;         // distance between two of its steps (= RG_CONSUMERS)
+    // (row block, step in row block) of this warp's current step, advanced without divisions
+    int64_t rb = g_begin / spr;
+    int c = (int)(g_begin - rb * spr) + j_first;
+    while (c >= spr) { c -= spr; ++rb; }
+    if (j_first < nsteps) load_scales(rb, c, 0);
+
+    pdl_wait();  // x, Y and the workspace may belong to the previous kernel in the stream
+    if constexpr (XSMEM) {
+        uint4* dst = reinterpret_cast<uint4*>(smem + 1024);
+        const uint4* src = reinterpret_cast<const uint4*>(X);
+        const int n16 = (int)((int64_t)M * K / 8);
+        for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) dst[i] = __ldg(src + i);
+        consumer_bar_sync();
+    }
+
+    // per-lane activation row pointers for the tensor path (token = 8*mt + gid), hoisted out of the loop
+    const uint4* xrow[MT];
+    bool xrow_ok[MT];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const int token = 8 * mt + gid;
+        xrow_ok[mt] = MMA && token < M;
+        xrow[mt] = (XSMEM ? xs : reinterpret_cast<const uint4*>(X)) + (xrow_ok[mt] ? (int64_t)token * (K / 8) : 0);
+    }
+    const int64_t rb_first = g_begin / spr;
+    for (int j2 = j_first; j2 < nsteps; j2 += 2 * J_STRIDE) {
+#pragma unroll
+      for (int buf = 0; buf < 2; ++buf) {  // two steps per trip so that the scale buffers are indexed statically
+        const int j = j2 + buf * J_STRIDE;
+        if (j >= nsteps) break;
+        int64_t rb_next = rb;
+        int c_next = c + J_STRIDE;
+        while (c_next >= spr) { c_next -= spr; ++rb_next; }
+        if (j + J_STRIDE < nsteps) load_scales(rb_next, c_next, buf ^ 1);
+        const int64_t cb = 4 * (int64_t)c + tig;
+        const bool valid = cb < ncb;
+        const int m = j / RG_Q;
+        const int slot = m % stages;
+        if (!mbar_wait(smem_u32(&bars[slot]), (uint32_t)((m / stages) & 1))) {
+            if (err && lane == 0) atomicCAS(err, 0, 2 | (m << 8) | (warp << 16) | (j << 24));
+        }
+        uint32_t rec[2][NW];
+        {
+            // records are fetched with lane (column block, row) = (lane / 8, lane % 8): 8 lanes read 128
+            // contiguous bytes, free of bank conflicts
+            const int ftig = lane >> 3, fgid = lane & 7;
+            const int64_t gs = g_begin + (int64_t)m * RG_Q;  // first step of this slot
+            const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - unit_index(gs) + ftig;
+            const bool fvalid = 4 * (int64_t)c + ftig < ncb;
+            const uint4* unit = reinterpret_cast<const uint4*>(ring + (size_t)slot * SLOT + uoff * UB);
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int t = 0; t < BITS; ++t) {
+                    uint4 q = make_uint4(0, 0, 0, 0);
+                    if (fvalid) q = unit[t * 16 + fgid + 8 * h];
+                    rec[h][4 * t + 0] = q.x; rec[h][4 * t + 1] = q.y; rec[h][4 * t + 2] = q.z; rec[h][4 * t + 3] = q.w;
+                }
+            if constexpr (MMA) {
+                // hand the records over to the lanes that own them in the MMA fragment layout
+                const int src = ((lane & 3) << 3) | (lane >> 2);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int i = 0; i < NW; ++i) rec[h][i] = __shfl_sync(0xffffffffu, rec[h][i], src);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
+
+        float acc[MMA ? 4 * MT : 4];
+#pragma unroll
+        for (int i = 0; i < (MMA ? 4 * MT : 4); ++i) acc[i] = 0.f;
+        if (!MMA) {
+            if (valid) {
+#pragma unroll
+                for (int T = 0; T < 4; ++T) {
+                    uint32_t xw[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 v = XSMEM ? xs[cb * 16 + 4 * T + i]
+                                              : __ldg(reinterpret_cast<const uint4*>(X) + cb * 16 + 4 * T + i);
+                        xw[4 * i + 0] = v.x; xw[4 * i + 1] = v.y; xw[4 * i + 2] = v.z; xw[4 * i + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t w2[16];
+                        if constexpr (!UNIFORM) {
+                            potl::pot_decode32<BITS>(rec[h], T, sc[buf][h][T >> 1], w2);
+                        } else {
+                            potl::UintParams pr;
+                            pr.s2 = potl::bits_h2(sc[buf][h][T >> 1]);
+                            pr.z = potl::bits_h2(zp[buf][h][T >> 1]);
+                            potl::uint_decode32<BITS>(rec[h], T, pr, w2);
+                        }
+#pragma unroll
+                        for (int p = 0; p < 16; ++p) rg_fma2(acc[2 * h], acc[2 * h + 1], w2[p], xw[p]);
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int T = 0; T < 4; ++T) {
+                uint32_t w0[16], w1[16];
+                potl::pot_decode32<BITS>(rec[0], T, sc[buf][0][T >> 1], w0);
+                potl::pot_decode32<BITS>(rec[1], T, sc[buf][1][T >> 1], w1);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    uint32_t xw[16];
+                    const bool xok = valid && xrow_ok[mt];
+                    const uint4* xp = xrow[mt] + cb * 16 + 4 * T;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (xok) v = XSMEM ? xp[i] : __ldg(xp + i);
+                        xw[4 * i + 0] = v.x; xw[4 * i + 1] = v.y; xw[4 * i + 2] = v.z; xw[4 * i + 3] = v.w;
+                    }
+                    float(&a)[4] = *reinterpret_cast<float(*)[4]>(&acc[4 * mt]);
+#pragma unroll
+                    for (int st = 0; st < 8; ++st)
+                        rg_mma(a, w0[2 * st], w1[2 * st], w0[2 * st + 1], w1[2 * st + 1], xw[2 * st], xw[2 * st + 1]);
+                }
+            }
+        }
+
+        // ---- deliver the step's partial sums -----------------------------------------------------------
+        // spr == 1: the step is the whole row block, write Y.  Otherwise the 16*TOK sums go to a slot:
+        // in shared memory when every step of the row block belongs to this CTA (the common case),
+        // else in the global workspace; whoever fills the last slot adds them in ascending column order.
+        const bool whole = (spr == 1);
+        const int64_t rb_g0 = rb * spr;  // first step of this row block
+        const bool local = cmb_bytes && rb_g0 >= g_begin && rb_g0 + spr <= g_end;
+        float* pslot = whole ? nullptr
+                            : (local ? cmb + (size_t)(rb_g0 - g_begin + c) * (16 * TOK)
+                                     : partial + (rb_g0 + c) * (16 * TOK));
+        if (!MMA) {
+            float r0 = acc[0] + acc[1], r1 = acc[2] + acc[3];
+            r0 += __shfl_xor_sync(0xffffffffu, r0, 8); r0 += __shfl_xor_sync(0xffffffffu, r0, 16);
+            r1 += __shfl_xor_sync(0xffffffffu, r1, 8); r1 += __shfl_xor_sync(0xffffffffu, r1, 16);
+            if (tig == 0) {
+                if (whole) {
+                    Y[rb * 16 + gid] = __float2half_rn(r0);
+                    Y[rb * 16 + gid + 8] = __float2half_rn(r1);
+                } else {
+                    pslot[gid] = r0;
+                    pslot[gid + 8] = r1;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int row = gid + 8 * (e >> 1), token = 8 * mt + 2 * tig + (e & 1);
+                    if (whole) {
+                        if (token < M) Y[(int64_t)token * N + rb * 16 + row] = __float2half_rn(acc[4 * mt + e]);
+                    } else {
+                        pslot[token * 16 + row] = acc[4 * mt + e];
+                    }
+                }
+        }
+        if (!whole) {
+            unsigned prev = 0;
+            if (local) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) prev = atomicAdd(&cmb_cnt[rb - rb_first], 1u);
+            } else {
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) prev = atomicAdd(&counters[rb], 1u);
+            }
+            prev = __shfl_sync(0xffffffffu, prev, 0);
+            if (prev == (unsigned)spr - 1u) {  // this warp delivered the last slot of the row block
+                if (local) __threadfence_block(); else __threadfence();
+                const float* first = local ? cmb + (size_t)(rb_g0 - g_begin) * (16 * TOK) : partial + rb_g0 * (16 * TOK);
+                for (int e = lane; e < 16 * TOK; e += 32) {
+                    const int row = e & 15, token = e >> 4;
+                    float sum = 0.f;
+                    if (local) {
+                        for (int q = 0; q < spr; ++q) sum += first[(size_t)q * (16 * TOK) + e];
+                    } else {
+                        for (int q = 0; q < spr; ++q) sum += __ldcg(first + (size_t)q * (16 * TOK) + e);
+                    }
+                    if (token < M) Y[(int64_t)token * N + rb * 16 + row] = __float2half_rn(sum);
+                }
+                if (!local && lane == 0) counters[rb] = 0u;  // leave the workspace ready for the next call
+            }
+        }
+        rb = rb_next;
+        c = c_next;
+      }
+    }
+}
+
+// Device error word shared by the ring kernels (0 = no bounded wait ever gave up).  One copy per
+// translation unit that includes this header; ring_error_ptr() returns this GPU's address of it.
+static __device__ int g_ring_error;
+inline int* ring_error_ptr() {
+    static std::atomic<int*> cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    int* p = cache[dev].load(std::memory_order_acquire);
+    if (!p) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_ring_error) != cudaSuccess) return nullptr;
+        p = (int*)q;
+        cache[dev].store(p, std::memory_order_release);
+    }
+    return p;
+}
+// Reads and clears the error word (synchronises the device).  -1 if it cannot be read.
+inline int ring_error_fetch() {
+    int v = -1, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_ring_error, sizeof(int)) != cudaSuccess) return -1;
+    cudaMemcpyToSymbol(g_ring_error, &zero, sizeof(int));
+    return v;
+}
+
+// Host side.  `err` may be nullptr.
+template <int BITS, int MODE, int MT>
+pot_status_t launch_ring(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
+                         const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
+    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1);
+    auto run = [&](auto kernel) -> pot_status_t {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
+            return POT_ERR_CUDA;
+        unsigned* counters = (unsigned*)workspace;
+        float* partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
+        return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(RG_THREADS), p.smem_bytes, s, (const uint4*)packed,
+                          (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
+                          (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
+    };
+    if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, true>);
+    return run(ring_kernel<BITS, MODE, MT, false>);
+}
+
+}  // namespace pot

@@ -40,11 +40,13 @@ def test_size_helpers(L):
     assert L.pot_scales_bytes(4096, 4096, 128) == 4096 * 32 * 2
     assert L.pot_scales_bytes(4096, 4096, 64) == 4096 * 64 * 2
     assert L.pot_scales_bytes(4096, 4096, 32) == 0
-    # big N alone fills the GPU: no split-K scratch; a short, wide matrix needs it
-    assert L.pot_gemv_workspace_bytes(12288, 4096, 3, 128) == 0
+    # one warp-step (512 columns) per row block: nothing to combine; longer rows need the step counters
+    # and one FP32 partial slot per (row block, step)
+    assert L.pot_gemv_workspace_bytes(12288, 512, 3, 128) == 0
     ws = L.pot_gemv_workspace_bytes(4096, 11008, 3, 128)
-    assert ws > 0 and ws % 16 == 0
-    assert L.pot_gemm_workspace_bytes(8, 12288, 4096, 3, 128) == 0
+    assert ws == 1024 + 256 * 22 * 16 * 4 and ws % 16 == 0
+    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
+    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 32 * 4
 
 
 def test_status_strings(L):
