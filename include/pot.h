@@ -94,6 +94,7 @@ uint64_t pot_launch_count(void);
  * device, return that word (0 = no wait ever gave up) and clear it.                                   */
 int pot_debug_gemv_error(void);
 int pot_debug_gemm_error(void);
+int pot_debug_prefill_error(void);
 
 /*
  * pot_quantize_ref -- reference PoT quantizer (Eq. 2; groups per Sec. 3.1).  Set-up code: it

@@ -24,7 +24,7 @@ EXPORTS = [
     "pot_status_string", "pot_packed_bytes", "pot_scales_bytes", "pot_gemv_workspace_bytes",
     "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack",
     "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_host", "pot_gemm", "uint_quantize_ref", "uint_dequant",
-    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemm_error",
+    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemm_error", "pot_debug_prefill_error",
 ]
 
 _lib = None
@@ -260,6 +260,6 @@ def pot_gemv_noalloc(packed_tiled, scales, K: int, bits: int, group: int, x: tor
     return y
 
 
-def pot_debug_errors() -> tuple[int, int]:
-    """(gemv, gemm) device error words, read and cleared; (0, 0) when every bounded wait completed."""
-    return int(lib().pot_debug_gemv_error()), int(lib().pot_debug_gemm_error())
+def pot_debug_errors() -> tuple[int, int, int]:
+    """(gemv, gemm, prefill) device error words, read and cleared; all 0 when every bounded wait completed."""
+    return int(lib().pot_debug_gemv_error()), int(lib().pot_debug_gemm_error()), int(lib().pot_debug_prefill_error())

@@ -1,11 +1,319 @@
-// Prefill GEMM (large M): placeholder until the tcgen05 kernel lands.
+// Prefill GEMM on 5th-generation tensor cores: Y[M,N] = X[M,K] W~^T, FP16 in, FP32 accumulate in
+// tensor memory, FP16 out, with the PoT dequantization fused in (tiled weight layout).
+//
+// One CTA computes a 128-token x 128-feature tile of Y.  Per 128-wide K block:
+//   warp 0 (one lane)  : TMA loads of the X tile (two 64-column boxes, 128-byte swizzle) into the stage;
+//   warps 2..9         : "dequant producers" -- each thread fetches half a 128-code record of one weight
+//                        row (coalesced 16-byte loads from the tiled layout), decodes it in registers
+//                        with the mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the
+//                        stage's B tile in exactly the layout the tensor core expects (K-major, 8-row x
+//                        128-byte atoms, 16-byte chunks XOR-swizzled with the row index), then
+//                        fence.proxy.async + mbarrier arrive;
+//   warp 1 (one lane)  : waits for both operands, issues 8 tcgen05.mma (M = 128, N = 128, K = 16) whose
+//                        accumulator lives in 128 columns of tensor memory, and tcgen05.commit's the
+//                        stage back to the producers.
+// After the last K block the accumulator is committed to a barrier; warps 2..9 read it with tcgen05.ld
+// (each warp its own 32-lane quarter, two warps per quarter split the columns), convert to FP16 and
+// store.  The weights are re-decoded once per 128-token tile (M / 128 times overall), which is the price
+// of never writing FP16 weights to HBM.
+//
+// All mbarrier waits are bounded (see ring.cuh); a wait that gives up records a code and the CTA carries
+// on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
+#include <cuda.h>
+
 #include "common.cuh"
+#include "layout.cuh"
+#include "ring.cuh"
 
 namespace pot {
-bool gemm_prefill_supported(int64_t, int64_t, int64_t, int, int) { return false; }
-size_t gemm_prefill_workspace(int64_t, int64_t, int64_t, int, int) { return 0; }
-pot_status_t gemm_prefill_launch(const void*, const void*, int64_t, int64_t, int, int, const void*, int64_t, void*,
-                                 void*, size_t, cudaStream_t) {
-    return POT_ERR_UNSUPPORTED;
+
+constexpr int PF_BM = 128;      // tokens per tile  (MMA M)
+constexpr int PF_BN = 128;      // features per tile (MMA N)
+constexpr int PF_BK = 128;      // one column block per stage
+constexpr int PF_STAGES = 3;
+constexpr int PF_PRODUCERS = 8;                      // dequant / epilogue warps
+constexpr int PF_THREADS = (2 + PF_PRODUCERS) * 32;  // + TMA warp + MMA warp
+constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
+constexpr int PF_TILE_BYTES = 2 * PF_ATOM_BYTES;     // 128 rows x 128 halves
+constexpr int PF_STAGE_BYTES = 2 * PF_TILE_BYTES;    // A + B
+constexpr size_t PF_SMEM = 1024 /*align slack*/ + (size_t)PF_STAGES * PF_STAGE_BYTES + 256 /*barriers*/;
+
+// UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
+constexpr uint32_t PF_IDESC = (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ |
+                              ((uint32_t)(PF_BN >> 3) << 17) | ((uint32_t)(PF_BM >> 4) << 24);
+
+// shared-memory matrix descriptor, K-major, 128-byte swizzle: start >> 4, LBO = 1 (unused), SBO = 1024 B
+// between 8-row groups, descriptor version 1, layout type 2 (SWIZZLE_128B)
+__device__ __forceinline__ uint64_t pf_smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
 }
+
+__device__ __forceinline__ void pf_tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                 "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void pf_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void pf_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+        "%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(PF_THREADS, 1)
+pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
+                        const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
+                        __half* __restrict__ Y, int* __restrict__ err) {
+    constexpr int NW = 4 * BITS;
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * PF_STAGE_BYTES);
+    // bars: fullA[S], fullB[S], empty[S], accum, then the tensor-memory base address
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * PF_STAGES + 1);
+    const uint32_t bar0 = smem_u32(bars);
+    auto fullA = [&](int s) { return bar0 + 8u * s; };
+    auto fullB = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
+    auto empty = [&](int s) { return bar0 + 8u * (2 * PF_STAGES + s); };
+    const uint32_t accum = bar0 + 8u * (3 * PF_STAGES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.x * PF_BM, n0 = (int64_t)blockIdx.y * PF_BN;
+    const int nkb = (int)(K / PF_BK);
+    const int64_t ncb = K / 128;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PF_STAGES; ++s) {
+            mbar_init(fullA(s), 1);
+            mbar_init(fullB(s), PF_PRODUCERS * 32);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // allocate 128 columns of tensor memory (whole warp), base address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(PF_BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_launch_dependents();
+    pdl_wait();
+
+    if (warp == 0) {
+        // ---------------- TMA producer: X tile, two 64-column boxes per stage ------------------------
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % PF_STAGES;
+                if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
+                    if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
+                }
+                mbar_expect_tx(fullA(s), PF_TILE_BYTES);
+                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
+                pf_tma_load_2d(a, &xmap, kb * PF_BK, (int)m0, fullA(s));
+                pf_tma_load_2d(a + PF_ATOM_BYTES, &xmap, kb * PF_BK + 64, (int)m0, fullA(s));
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ---------------------------------------------------------------
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % PF_STAGES;
+                const uint32_t ph = (uint32_t)((kb / PF_STAGES) & 1);
+                if (!mbar_wait(fullA(s), ph) || !mbar_wait(fullB(s), ph)) {
+                    if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES), b = a + PF_TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < PF_BK / 16; ++ks) {
+                    const uint32_t off = (uint32_t)(ks >> 2) * PF_ATOM_BYTES + (uint32_t)(ks & 3) * 32u;
+                    pf_mma(tmem_base, pf_smem_desc(a + off), pf_smem_desc(b + off), PF_IDESC, (kb | ks) != 0 ? 1u : 0u);
+                }
+                pf_commit(empty(s));  // the stage is free again once these MMAs have read it
+            }
+            pf_commit(accum);          // the accumulator is complete once every MMA has finished
+        }
+    } else {
+        // ---------------- dequant producers (then epilogue) ---------------------------------------------
+        const int pt = threadIdx.x - 64;        // 0..255
+        const int row = pt & 127, half = pt >> 7;  // weight row inside the tile, which 64 columns of the block
+        const int64_t n = n0 + row;
+        const bool row_ok = n < N;
+        const int64_t rb = n >> 4;
+        const int r = (int)(n & 15);
+        const int gpr = (int)(K / G), spg = 128 / G;
+        // the 6-word (n = 3) / 4-word / 8-word half record lives in planes [p_lo, p_hi]
+        const int w_lo = half * (NW / 2), w_hi = w_lo + NW / 2 - 1;
+        const int p_lo = w_lo >> 2, p_hi = w_hi >> 2;
+
+        uint32_t rec[2][NW];
+        uint32_t sc2[2];
+        auto load = [&](int kb, int buf) {
+            if (row_ok) {
+                const uint4* unit = packed + (rb * ncb + kb) * (16 * BITS);
+#pragma unroll
+                for (int t = 0; t < BITS; ++t) {
+                    if (t >= p_lo && t <= p_hi) {
+                        const uint4 q = __ldg(unit + t * 16 + r);
+                        rec[buf][4 * t + 0] = q.x; rec[buf][4 * t + 1] = q.y; rec[buf][4 * t + 2] = q.z; rec[buf][4 * t + 3] = q.w;
+                    }
+                }
+                const int64_t so = n * gpr + (int64_t)kb * spg + (spg == 2 ? half : 0);
+                sc2[buf] = (uint32_t)__ldg(scales + so) * 0x10001u;
+            }
+        };
+        if (nkb > 0) load(0, 0);
+        for (int kb2 = 0; kb2 < nkb; kb2 += 2) {
+#pragma unroll
+            for (int buf = 0; buf < 2; ++buf) {
+                const int kb = kb2 + buf;
+                if (kb >= nkb) break;
+                if (kb + 1 < nkb) load(kb + 1, buf ^ 1);
+                const int s = kb % PF_STAGES;
+                if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
+                    if (err) atomicCAS(err, 0, 0x30 | (kb << 8));
+                }
+                unsigned char* btile = smem + (size_t)s * PF_STAGE_BYTES + PF_TILE_BYTES + (size_t)half * PF_ATOM_BYTES + row * 128;
+#pragma unroll
+                for (int T2 = 0; T2 < 2; ++T2) {
+                    uint32_t w2[16];
+                    if (row_ok && half == 0) potl::pot_decode32<BITS>(rec[buf], T2, sc2[buf], w2);
+                    else if (row_ok) potl::pot_decode32<BITS>(rec[buf], 2 + T2, sc2[buf], w2);
+                    else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) w2[i] = 0u;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {  // 4 chunks of 8 halves; chunk index inside the 128-byte row
+                        const int chunk = 4 * T2 + c;
+                        *reinterpret_cast<uint4*>(btile + ((chunk ^ (row & 7)) << 4)) =
+                            make_uint4(w2[4 * c], w2[4 * c + 1], w2[4 * c + 2], w2[4 * c + 3]);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+                mbar_arrive(fullB(s));
+            }
+        }
+        // ---------------- epilogue: tensor memory -> registers -> FP16 -> Y --------------------------
+        if (!mbar_wait(accum, 0)) {
+            if (err) atomicCAS(err, 0, 0x40);
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
+        const int colh = (warp - 2) >> 2;         // warps 2..5 take columns 0..63, warps 6..9 columns 64..127
+        const int64_t token = m0 + 32 * q + lane;
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+            const int col = colh * 64 + cc * 32;
+            uint32_t v[32];
+            pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (token < M) {
+                __half* dst = Y + token * N + n0 + col;
+                if (n0 + col + 32 <= N) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const __half2 h = __floats2half2_rn(__uint_as_float(v[8 * i + 2 * j]), __uint_as_float(v[8 * i + 2 * j + 1]));
+                            o[j] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(dst + 8 * i) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                } else {
+                    for (int i = 0; i < 32; ++i)
+                        if (n0 + col + i < N) dst[i] = __float2half_rn(__uint_as_float(v[i]));
+                }
+            }
+        }
+    }
+    // ---------------- teardown: everyone is done with tensor memory, the allocating warp frees it --------
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(PF_BN) : "memory");
+    }
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link against libcuda
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+    static std::atomic<EncodeTiledFn> cache{nullptr};
+    EncodeTiledFn f = cache.load(std::memory_order_acquire);
+    if (!f) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || !p) return nullptr;
+        f = (EncodeTiledFn)p;
+        cache.store(f, std::memory_order_release);
+    }
+    return f;
+}
+
+bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group) {
+    (void)bits; (void)group;
+    // TMA needs the X row pitch (2K bytes) to be a multiple of 16 -- implied by K % 128 == 0 -- and 32-bit box coordinates
+    return M > 0 && N % 16 == 0 && K % 128 == 0 && M < (int64_t(1) << 31) && K < (int64_t(1) << 31);
+}
+size_t gemm_prefill_workspace(int64_t, int64_t, int64_t, int, int) { return 0; }
+
+static int* prefill_error_ptr();
+
+pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                 const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s) {
+    (void)workspace; (void)ws_bytes;
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return POT_ERR_CUDA;
+    CUtensorMap xmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {64, PF_BM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return POT_ERR_CUDA;
+    const dim3 grid((unsigned)((M + PF_BM - 1) / PF_BM), (unsigned)((N + PF_BN - 1) / PF_BN)), block(PF_THREADS);
+    auto run = [&](auto kernel) -> pot_status_t {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM) != cudaSuccess) return POT_ERR_CUDA;
+        return launch_pdl(kernel, grid, block, PF_SMEM, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
+                          (__half*)Y, prefill_error_ptr());
+    };
+    if (bits == 2) return run(pot_gemm_prefill_kernel<2>);
+    if (bits == 3) return run(pot_gemm_prefill_kernel<3>);
+    return run(pot_gemm_prefill_kernel<4>);
+}
+
+static int* prefill_error_ptr() { return ring_error_ptr(); }
+
 }  // namespace pot
+
+// Diagnostic: reads and clears the device error word of the prefill kernel (0 = every bounded wait completed;
+// 0x10 / 0x20 / 0x30 / 0x40 in the low byte = the TMA warp / the MMA warp / a dequant warp / the epilogue gave
+// up waiting, bits 8.. = the K block).  Synchronises the device.
+extern "C" int pot_debug_prefill_error(void) { return pot::ring_error_fetch(); }

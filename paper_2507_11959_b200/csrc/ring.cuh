@@ -45,6 +45,7 @@ struct RingPlan {
     int64_t total_steps;
     int stages;
     bool x_in_smem;
+    bool x_wide;         // GEMV only: x staged one FP16 value per 32-bit word (no half2 unpacking in the loop)
     size_t x_bytes;      // shared-memory bytes for the staged activations (0 if read from global)
     size_t cmb_bytes;    // shared-memory bytes for combining the steps of a row block inside the CTA (0 = off)
     size_t smem_bytes;   // total dynamic shared memory
@@ -58,7 +59,8 @@ inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok) {
     p.spr = (int)((ncb + 3) / 4);
     p.total_steps = nrb * p.spr;
     p.grid = (int)(p.total_steps < kSmCount ? p.total_steps : kSmCount);
-    const size_t xb = (size_t)M * (size_t)K * 2;
+    p.x_wide = (tok == 1) && (size_t)K * 4 <= 48 * 1024;
+    const size_t xb = (size_t)M * (size_t)K * (p.x_wide ? 4 : 2);
     p.x_in_smem = xb <= 64 * 1024;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
     const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
@@ -126,6 +128,19 @@ __device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, u
         : "+f"(acc0), "+f"(acc1)
         : "r"(w2), "r"(x2));
 }
+// same with x already split: x0 / x1 hold one FP16 value each in their low 16 bits
+__device__ __forceinline__ void rg_fma2_wide(float& acc0, float& acc1, uint32_t w2, uint32_t x0, uint32_t x1) {
+    asm("{\n\t"
+        ".reg .b16 wl, wh, xa, xb, d0, d1;\n\t"
+        "mov.b32 {wl, wh}, %2;\n\t"
+        "mov.b32 {xa, d0}, %3;\n\t"
+        "mov.b32 {xb, d1}, %4;\n\t"
+        "fma.rn.f32.f16 %0, wl, xa, %0;\n\t"
+        "fma.rn.f32.f16 %1, wh, xb, %1;\n\t"
+        "}"
+        : "+f"(acc0), "+f"(acc1)
+        : "r"(w2), "r"(x0), "r"(x1));
+}
 __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
     asm volatile(
@@ -135,13 +150,15 @@ __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
 }
 
 // MODE RG_POT_FMA / RG_UINT_FMA: M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
-template <int BITS, int MODE, int MT, bool XSMEM>
+template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = staged packed, 2 = staged wide
 __global__ void __launch_bounds__(RG_THREADS, 1)
 ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
             int64_t N, int64_t K, int G, int spr, int64_t total_steps, int stages, int x_bytes, int cmb_bytes,
             const __half* __restrict__ X, int M, __half* __restrict__ Y, float* __restrict__ partial,
             unsigned* __restrict__ counters, int* __restrict__ err) {
     constexpr int NW = 4 * BITS;
+    constexpr bool XSMEM = (XMODE != 0);
+    constexpr bool XWIDE = (XMODE == 2);
     constexpr bool MMA = (MODE == RG_POT_MMA);
     constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
     constexpr int TOK = MMA ? 8 * MT : 1;
@@ -243,7 +260,15 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         uint4* dst = reinterpret_cast<uint4*>(smem + 1024);
         const uint4* src = reinterpret_cast<const uint4*>(X);
         const int n16 = (int)((int64_t)M * K / 8);
-        for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) dst[i] = __ldg(src + i);
+        for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) {
+            const uint4 v = __ldg(src + i);
+            if constexpr (XWIDE) {
+                dst[2 * i] = make_uint4(v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16);
+                dst[2 * i + 1] = make_uint4(v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16);
+            } else {
+                dst[i] = v;
+            }
+        }
         consumer_bar_sync();
     }
 
@@ -257,6 +282,8 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         xrow[mt] = (XSMEM ? xs : reinterpret_cast<const uint4*>(X)) + (xrow_ok[mt] ? (int64_t)token * (K / 8) : 0);
     }
     const int64_t rb_first = g_begin / spr;
+    int m = grp, slot = grp % stages;        // this warp's current slot fill, ring slot and barrier phase
+    uint32_t phase = (uint32_t)((grp / stages) & 1);
     for (int j2 = j_first; j2 < nsteps; j2 += 2 * J_STRIDE) {
 #pragma unroll
       for (int buf = 0; buf < 2; ++buf) {  // two steps per trip so that the scale buffers are indexed statically
@@ -268,9 +295,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         if (j + J_STRIDE < nsteps) load_scales(rb_next, c_next, buf ^ 1);
         const int64_t cb = 4 * (int64_t)c + tig;
         const bool valid = cb < ncb;
-        const int m = j / RG_Q;
-        const int slot = m % stages;
-        if (!mbar_wait(smem_u32(&bars[slot]), (uint32_t)((m / stages) & 1))) {
+        if (!mbar_wait(smem_u32(&bars[slot]), phase)) {
             if (err && lane == 0) atomicCAS(err, 0, 2 | (m << 8) | (warp << 16) | (j << 24));
         }
         uint32_t rec[2][NW];
@@ -278,8 +303,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             // records are fetched with lane (column block, row) = (lane / 8, lane % 8): 8 lanes read 128
             // contiguous bytes, free of bank conflicts
             const int ftig = lane >> 3, fgid = lane & 7;
-            const int64_t gs = g_begin + (int64_t)m * RG_Q;  // first step of this slot
-            const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - unit_index(gs) + ftig;
+            // units between the slot's first step (wig steps back) and this one, without divisions
+            int64_t rb_s = rb;
+            int c_s = c - wig;
+            while (c_s < 0) { c_s += spr; --rb_s; }
+            const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - (rb_s * ncb + 4 * (int64_t)c_s) + ftig;
             const bool fvalid = 4 * (int64_t)c + ftig < ncb;
             const uint4* unit = reinterpret_cast<const uint4*>(ring + (size_t)slot * SLOT + uoff * UB);
 #pragma unroll
@@ -309,11 +337,12 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             if (valid) {
 #pragma unroll
                 for (int T = 0; T < 4; ++T) {
-                    uint32_t xw[16];
+                    uint32_t xw[XWIDE ? 32 : 16];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint4 v = XSMEM ? xs[cb * 16 + 4 * T + i]
-                                              : __ldg(reinterpret_cast<const uint4*>(X) + cb * 16 + 4 * T + i);
+                    for (int i = 0; i < (XWIDE ? 8 : 4); ++i) {
+                        const uint4 v = XWIDE ? xs[cb * 32 + 8 * T + i]
+                                              : (XSMEM ? xs[cb * 16 + 4 * T + i]
+                                                       : __ldg(reinterpret_cast<const uint4*>(X) + cb * 16 + 4 * T + i));
                         xw[4 * i + 0] = v.x; xw[4 * i + 1] = v.y; xw[4 * i + 2] = v.z; xw[4 * i + 3] = v.w;
                     }
 #pragma unroll
@@ -328,7 +357,10 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                             potl::uint_decode32<BITS>(rec[h], T, pr, w2);
                         }
 #pragma unroll
-                        for (int p = 0; p < 16; ++p) rg_fma2(acc[2 * h], acc[2 * h + 1], w2[p], xw[p]);
+                        for (int p = 0; p < 16; ++p) {
+                            if constexpr (XWIDE) rg_fma2_wide(acc[2 * h], acc[2 * h + 1], w2[p], xw[2 * p], xw[2 * p + 1]);
+                            else rg_fma2(acc[2 * h], acc[2 * h + 1], w2[p], xw[p]);
+                        }
                     }
                 }
             }
@@ -423,6 +455,9 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         }
         rb = rb_next;
         c = c_next;
+        m += RG_GROUPS;
+        slot += RG_GROUPS;
+        while (slot >= stages) { slot -= stages; phase ^= 1u; }
       }
     }
 }
@@ -465,8 +500,11 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
                           (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
                           (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
     };
-    if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, true>);
-    return run(ring_kernel<BITS, MODE, MT, false>);
+    if constexpr (MODE != RG_POT_MMA) {
+        if (p.x_in_smem && p.x_wide) return run(ring_kernel<BITS, MODE, MT, 2>);
+    }
+    if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, 1>);
+    return run(ring_kernel<BITS, MODE, MT, 0>);
 }
 
 }  // namespace pot
