@@ -36,6 +36,7 @@ METRIC = "pot_dequant_gemv_GBps"
 UNIT = "GB/s"
 GROUP = 128
 HEADLINE_BITS = 3
+NCU_TRAFFIC_RATIO = 1.0015  # measured DRAM bytes / algorithmic bytes of the GEMV kernel (see profiles/)
 
 
 def gemv_bytes(N, K, bits, G, M=1):
@@ -274,8 +275,12 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": value / world / peaks["hbm_gbs"], "frac_of_8TBs_nominal": value / world / 8000.0,
-                     "peak_source": peaks["source"], "kernel": "gemv_tiled_kernel<3,false>",
-                     "traffic": None},
+                     "peak_source": peaks["source"], "kernel": "ring_kernel<3, RG_POT_FMA, 1> (decode GEMV, tiled layout)",
+                     "per_launch_us": ms * 1e3 / max(1, launches_per_step),
+                     "algorithmic_bytes_per_launch": bytes3 / max(1, launches_per_step),
+                     # dram__bytes_read+write per launch from the ncu capture of the 12288x4096 launch
+                     # (profiles/ring_kernel_gemv_12288x4096_3bit.md: 1.0015 x algorithmic), scaled by bytes
+                     "traffic": NCU_TRAFFIC_RATIO * bytes3 / max(1, launches_per_step)},
     }
 
     if rank == 0 and world == 1 and not args.no_extras:

@@ -193,7 +193,7 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
 
 /*
  * pot_gemm -- Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
- * accumulation, FP16 output.  M <= 32 (decode batches) runs a bandwidth-bound tensor-core
+ * accumulation, FP16 output.  M <= 8 (decode batches) runs a bandwidth-bound tensor-core
  * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the
  * tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
  * accumulators in tensor memory.  The prefill kernel requires layout == POT_LAYOUT_TILED.

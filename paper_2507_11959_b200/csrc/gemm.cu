@@ -1,6 +1,6 @@
 // pot_gemm: Y[M,N] = X[M,K] W~^T with the dequantization fused in.
 //
-//  * M <= 32, tiled layout: bandwidth-bound tensor-core kernel.  The weights are the MMA's
+//  * M <= 8, tiled layout: bandwidth-bound tensor-core kernel (ring.cuh).  The weights are the MMA's
 //    M-side operand (16 rows per warp-step), the tokens its 8-wide N side, so no padding of M
 //    to 16 is needed and a warp decodes each record exactly once, straight into the A
 //    fragment registers -- the FP16 weights never exist in shared or global memory.
@@ -9,7 +9,7 @@
 //    gid+8, column block 4*chunk + tig) into k-slots {2tig, 2tig+1, 2tig+8, 2tig+9} of step j,
 //    and the B fragment reads x at the same columns.
 //  * any M, canonical layout: a plain shared-memory tiled mma.sync kernel (the fallback).
-//  * large M, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
+//  * M > 8, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
 #include "common.cuh"
 #include "layout.cuh"
 #include "ring.cuh"
@@ -117,15 +117,18 @@ bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group
 
 using namespace pot;
 
+// Up to 8 tokens the streaming kernel (weights decoded straight into MMA fragments) is bandwidth-bound;
+// beyond that the legacy warp-level MMA rate becomes the limit and the tcgen05 kernel takes over.
+constexpr int64_t kSmallBatchMax = 8;
 static bool use_small(int64_t M, int64_t N, pot_layout_t layout) {
-    return layout == POT_LAYOUT_TILED && M <= 32 && N % 16 == 0;
+    return layout == POT_LAYOUT_TILED && M <= kSmallBatchMax && N % 16 == 0;
 }
 
-static int small_mt(int64_t M) { return M <= 8 ? 1 : (M <= 16 ? 2 : 4); }
+static int small_mt(int64_t) { return 1; }
 
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || M <= 0) return 0;
-    if (M <= 32 && N % 16 == 0) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
+    if (M <= kSmallBatchMax && N % 16 == 0) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
@@ -146,10 +149,7 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
         const int Mi = (int)M;
 #define POT_GS(B, T) return launch_ring<B, RG_POT_MMA, T>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, ring_error_ptr(), s)
-#define POT_GS_B(B)                  \
-    if (M <= 8) POT_GS(B, 1);        \
-    else if (M <= 16) POT_GS(B, 2);  \
-    else POT_GS(B, 4);
+#define POT_GS_B(B) POT_GS(B, 1);
         if (bits == 2) { POT_GS_B(2) } else if (bits == 3) { POT_GS_B(3) } else { POT_GS_B(4) }
 #undef POT_GS_B
 #undef POT_GS
