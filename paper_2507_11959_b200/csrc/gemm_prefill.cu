@@ -1,21 +1,22 @@
 // Prefill GEMM on 5th-generation tensor cores: Y[M,N] = X[M,K] W~^T, FP16 in, FP32 accumulate in
 // tensor memory, FP16 out, with the PoT dequantization fused in (tiled weight layout).
 //
-// One CTA computes a 128-token x 128-feature tile of Y.  Per 128-wide K block:
-//   warp 0 (one lane)  : TMA loads of the X tile (two 64-column boxes, 128-byte swizzle) into the stage;
-//   warps 2..9         : "dequant producers" -- each thread fetches half a 128-code record of one weight
-//                        row (coalesced 16-byte loads from the tiled layout), decodes it in registers
+// One CTA computes a 256-token x 128-feature tile of Y as two 128 x 128 accumulators that share every
+// decoded weight tile.  Per 64-wide K block (one pipeline stage, 48 KB):
+//   warp 0 (one lane)  : TMA loads of the two X tiles (64-column boxes, 128-byte swizzle) into the stage;
+//   warps 2..9         : "dequant producers" -- each thread fetches the 32 codes of one weight row that the
+//                        stage needs (16-byte loads from the tiled layout), decodes them in registers
 //                        with the mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the
 //                        stage's B tile in exactly the layout the tensor core expects (K-major, 8-row x
 //                        128-byte atoms, 16-byte chunks XOR-swizzled with the row index), then
 //                        fence.proxy.async + mbarrier arrive;
-//   warp 1 (one lane)  : waits for both operands, issues 8 tcgen05.mma (M = 128, N = 128, K = 16) whose
-//                        accumulator lives in 128 columns of tensor memory, and tcgen05.commit's the
+//   warp 1 (one lane)  : waits for both operands, issues 2 x 4 tcgen05.mma (M = 128, N = 128, K = 16) whose
+//                        accumulators live in 2 x 128 columns of tensor memory, and tcgen05.commit's the
 //                        stage back to the producers.
-// After the last K block the accumulator is committed to a barrier; warps 2..9 read it with tcgen05.ld
-// (each warp its own 32-lane quarter, two warps per quarter split the columns), convert to FP16 and
-// store.  The weights are re-decoded once per 128-token tile (M / 128 times overall), which is the price
-// of never writing FP16 weights to HBM.
+// After the last K block the accumulators are committed to a barrier; warps 2..9 read them with
+// tcgen05.ld (each warp its own 32-lane quarter of one accumulator), convert to FP16 and store.  The
+// weights are re-decoded once per 256-token tile (M / 256 times overall), which is the price of never
+// writing FP16 weights to HBM.
 //
 // All mbarrier waits are bounded (see ring.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
@@ -27,16 +28,15 @@
 
 namespace pot {
 
-constexpr int PF_BM = 128;      // tokens per tile  (MMA M)
+constexpr int PF_BM = 128;      // tokens per accumulator (MMA M)
+constexpr int PF_MT = 2;        // accumulators per CTA: 256 tokens share one decoded weight tile
 constexpr int PF_BN = 128;      // features per tile (MMA N)
-constexpr int PF_BK = 128;      // one column block per stage
-constexpr int PF_STAGES = 3;
+constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte swizzle atom wide)
 constexpr int PF_PRODUCERS = 8;                      // dequant / epilogue warps
 constexpr int PF_THREADS = (2 + PF_PRODUCERS) * 32;  // + TMA warp + MMA warp
 constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
-constexpr int PF_TILE_BYTES = 2 * PF_ATOM_BYTES;     // 128 rows x 128 halves
-constexpr int PF_STAGE_BYTES = 2 * PF_TILE_BYTES;    // A + B
-constexpr size_t PF_SMEM = 1024 /*align slack*/ + (size_t)PF_STAGES * PF_STAGE_BYTES + 256 /*barriers*/;
+constexpr int PF_STAGE_BYTES = (PF_MT + 1) * PF_ATOM_BYTES;  // two X tiles + one weight tile
+constexpr size_t pf_smem_bytes(int stages) { return 1024 /*align slack*/ + (size_t)stages * PF_STAGE_BYTES + 256 /*barriers*/; }
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
 constexpr uint32_t PF_IDESC = (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ |
@@ -77,8 +77,10 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "memory");
 }
 
-template <int BITS>
-__global__ void __launch_bounds__(PF_THREADS, 1)
+// PF_STAGES = 2: two CTAs share an SM and hide each other's hand-off latencies (large M, many tiles);
+// PF_STAGES = 4: one CTA per SM with a deeper pipeline (few tiles, e.g. decode batches of 9..256 tokens).
+template <int BITS, int PF_STAGES>
+__global__ void __launch_bounds__(PF_THREADS, PF_STAGES == 2 ? 2 : 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
                         __half* __restrict__ Y, int* __restrict__ err) {
@@ -96,21 +98,21 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const uint32_t accum = bar0 + 8u * (3 * PF_STAGES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * PF_BM, n0 = (int64_t)blockIdx.y * PF_BN;
+    const int64_t m0 = (int64_t)blockIdx.x * (PF_BM * PF_MT), n0 = (int64_t)blockIdx.y * PF_BN;
     const int nkb = (int)(K / PF_BK);
     const int64_t ncb = K / 128;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
             mbar_init(fullA(s), 1);
-            mbar_init(fullB(s), PF_PRODUCERS * 32);
+            mbar_init(fullB(s), PF_PRODUCERS);   // one arrival per producer warp
             mbar_init(empty(s), 1);
         }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {  // allocate 128 columns of tensor memory (whole warp), base address lands in shared memory
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(PF_BN) : "memory");
+    if (warp == 1) {  // allocate 256 columns of tensor memory (whole warp), base address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(PF_BN * PF_MT) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -121,17 +123,18 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     pdl_wait();
 
     if (warp == 0) {
-        // ---------------- TMA producer: X tile, two 64-column boxes per stage ------------------------
+        // ---------------- TMA producer: two X tiles (64 columns x 128 tokens each) per stage --------------
         if (lane == 0) {
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % PF_STAGES;
                 if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
                 }
-                mbar_expect_tx(fullA(s), PF_TILE_BYTES);
+                mbar_expect_tx(fullA(s), PF_MT * PF_ATOM_BYTES);
                 const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
-                pf_tma_load_2d(a, &xmap, kb * PF_BK, (int)m0, fullA(s));
-                pf_tma_load_2d(a + PF_ATOM_BYTES, &xmap, kb * PF_BK + 64, (int)m0, fullA(s));
+#pragma unroll
+                for (int mt = 0; mt < PF_MT; ++mt)
+                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, kb * PF_BK, (int)m0 + mt * PF_BM, fullA(s));
             }
         }
     } else if (warp == 1) {
@@ -144,75 +147,84 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
                 }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES), b = a + PF_TILE_BYTES;
+                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES), b = a + PF_MT * PF_ATOM_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < PF_BK / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(ks >> 2) * PF_ATOM_BYTES + (uint32_t)(ks & 3) * 32u;
-                    pf_mma(tmem_base, pf_smem_desc(a + off), pf_smem_desc(b + off), PF_IDESC, (kb | ks) != 0 ? 1u : 0u);
-                }
+                for (int mt = 0; mt < PF_MT; ++mt)
+#pragma unroll
+                    for (int ks = 0; ks < PF_BK / 16; ++ks)
+                        pf_mma(tmem_base + (uint32_t)(mt * PF_BN), pf_smem_desc(a + mt * PF_ATOM_BYTES + ks * 32),
+                               pf_smem_desc(b + ks * 32), PF_IDESC, (kb | ks) != 0 ? 1u : 0u);
                 pf_commit(empty(s));  // the stage is free again once these MMAs have read it
             }
-            pf_commit(accum);          // the accumulator is complete once every MMA has finished
+            pf_commit(accum);          // the accumulators are complete once every MMA has finished
         }
     } else {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
-        const int pt = threadIdx.x - 64;        // 0..255
-        const int row = pt & 127, half = pt >> 7;  // weight row inside the tile, which 64 columns of the block
+        const int pt = threadIdx.x - 64;            // 0..255
+        const int row = pt & 127, qsel = pt >> 7;   // weight row inside the tile; which 32 of the stage's 64 columns
         const int64_t n = n0 + row;
         const bool row_ok = n < N;
         const int64_t rb = n >> 4;
         const int r = (int)(n & 15);
         const int gpr = (int)(K / G), spg = 128 / G;
-        // the 6-word (n = 3) / 4-word / 8-word half record lives in planes [p_lo, p_hi]
-        const int w_lo = half * (NW / 2), w_hi = w_lo + NW / 2 - 1;
-        const int p_lo = w_lo >> 2, p_hi = w_hi >> 2;
 
-        uint32_t rec[2][NW];
-        uint32_t sc2[2];
+        // stage kb covers columns 64*kb .. 64*kb+63 = quarter-records T = 2*(kb&1) + qsel of column block kb/2
+        // The packed codes are prefetched PF_DEPTH - 1 stages ahead (a stage lasts less than a memory latency).
+        constexpr int PF_DEPTH = 4;
+        uint32_t rec[PF_DEPTH][NW];
+        uint32_t sc2[PF_DEPTH];
         auto load = [&](int kb, int buf) {
             if (row_ok) {
-                const uint4* unit = packed + (rb * ncb + kb) * (16 * BITS);
+                const int T = 2 * (kb & 1) + qsel;
+                const int w_lo = T * (NW / 4), w_hi = w_lo + NW / 4 - 1;   // the quarter record's words
+                const uint4* unit = packed + (rb * ncb + (kb >> 1)) * (16 * BITS);
 #pragma unroll
                 for (int t = 0; t < BITS; ++t) {
-                    if (t >= p_lo && t <= p_hi) {
+                    if (t >= (w_lo >> 2) && t <= (w_hi >> 2)) {
                         const uint4 q = __ldg(unit + t * 16 + r);
                         rec[buf][4 * t + 0] = q.x; rec[buf][4 * t + 1] = q.y; rec[buf][4 * t + 2] = q.z; rec[buf][4 * t + 3] = q.w;
                     }
                 }
-                const int64_t so = n * gpr + (int64_t)kb * spg + (spg == 2 ? half : 0);
-                sc2[buf] = (uint32_t)__ldg(scales + so) * 0x10001u;
+                const int64_t so = n * gpr + (int64_t)(kb >> 1) * spg + (spg == 2 ? (kb & 1) : 0);
+                sc2[buf] = (uint32_t)__ldg(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
-        if (nkb > 0) load(0, 0);
-        for (int kb2 = 0; kb2 < nkb; kb2 += 2) {
 #pragma unroll
-            for (int buf = 0; buf < 2; ++buf) {
-                const int kb = kb2 + buf;
+        for (int p = 0; p < PF_DEPTH - 1; ++p)
+            if (p < nkb) load(p, p);
+        for (int kb4 = 0; kb4 < nkb; kb4 += PF_DEPTH) {
+#pragma unroll
+            for (int buf = 0; buf < PF_DEPTH; ++buf) {
+                const int kb = kb4 + buf;
                 if (kb >= nkb) break;
-                if (kb + 1 < nkb) load(kb + 1, buf ^ 1);
+                if (kb + PF_DEPTH - 1 < nkb) load(kb + PF_DEPTH - 1, (buf + PF_DEPTH - 1) % PF_DEPTH);
                 const int s = kb % PF_STAGES;
-                if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
-                    if (err) atomicCAS(err, 0, 0x30 | (kb << 8));
+                if (kb >= PF_STAGES) {  // one lane polls for the whole warp: the warp is about to WRITE the stage
+                    if (lane == 0 && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
+                        if (err) atomicCAS(err, 0, 0x30 | (kb << 8));
+                    }
+                    __syncwarp();
                 }
-                unsigned char* btile = smem + (size_t)s * PF_STAGE_BYTES + PF_TILE_BYTES + (size_t)half * PF_ATOM_BYTES + row * 128;
+                uint32_t w2[16];
+                if (row_ok) {
+                    // buf has the parity of kb, so the quarter index 2*(kb&1) + qsel is static in each branch
+                    const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
+                    if (qsel == 0) potl::pot_decode32<BITS>(rec[buf], 2 * (buf & 1), s2, w2);
+                    else potl::pot_decode32<BITS>(rec[buf], 2 * (buf & 1) + 1, s2, w2);
+                } else {
 #pragma unroll
-                for (int T2 = 0; T2 < 2; ++T2) {
-                    uint32_t w2[16];
-                    if (row_ok && half == 0) potl::pot_decode32<BITS>(rec[buf], T2, sc2[buf], w2);
-                    else if (row_ok) potl::pot_decode32<BITS>(rec[buf], 2 + T2, sc2[buf], w2);
-                    else {
+                    for (int i = 0; i < 16; ++i) w2[i] = 0u;
+                }
+                unsigned char* brow = smem + (size_t)s * PF_STAGE_BYTES + PF_MT * PF_ATOM_BYTES + row * 128;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) w2[i] = 0u;
-                    }
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {  // 4 chunks of 8 halves; chunk index inside the 128-byte row
-                        const int chunk = 4 * T2 + c;
-                        *reinterpret_cast<uint4*>(btile + ((chunk ^ (row & 7)) << 4)) =
-                            make_uint4(w2[4 * c], w2[4 * c + 1], w2[4 * c + 2], w2[4 * c + 3]);
-                    }
+                for (int c = 0; c < 4; ++c) {  // 4 chunks of 8 halves; chunk index inside the 128-byte row
+                    const int chunk = 4 * qsel + c;
+                    *reinterpret_cast<uint4*>(brow + ((chunk ^ (row & 7)) << 4)) =
+                        make_uint4(w2[4 * c], w2[4 * c + 1], w2[4 * c + 2], w2[4 * c + 3]);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
-                mbar_arrive(fullB(s));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(fullB(s));
             }
         }
         // ---------------- epilogue: tensor memory -> registers -> FP16 -> Y --------------------------
@@ -221,13 +233,13 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
-        const int colh = (warp - 2) >> 2;         // warps 2..5 take columns 0..63, warps 6..9 columns 64..127
-        const int64_t token = m0 + 32 * q + lane;
+        const int mt = (warp - 2) >> 2;           // warps 2..5 read accumulator 0, warps 6..9 accumulator 1
+        const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-            const int col = colh * 64 + cc * 32;
+        for (int cc = 0; cc < PF_BN / 32; ++cc) {
+            const int col = cc * 32;
             uint32_t v[32];
-            pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
+            pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(mt * PF_BN + col), v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             if (token < M) {
                 __half* dst = Y + token * N + n0 + col;
@@ -254,7 +266,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(PF_BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(PF_BN * PF_MT) : "memory");
     }
 }
 
@@ -298,15 +310,22 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
-    const dim3 grid((unsigned)((M + PF_BM - 1) / PF_BM), (unsigned)((N + PF_BN - 1) / PF_BN)), block(PF_THREADS);
-    auto run = [&](auto kernel) -> pot_status_t {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM) != cudaSuccess) return POT_ERR_CUDA;
-        return launch_pdl(kernel, grid, block, PF_SMEM, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
+    const dim3 grid((unsigned)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)), (unsigned)((N + PF_BN - 1) / PF_BN)), block(PF_THREADS);
+    const bool deep = (int64_t)grid.x * grid.y <= 2 * kSmCount;  // too few tiles to fill two CTAs per SM anyway
+    auto run = [&](auto kernel, int stages) -> pot_status_t {
+        const size_t smem = pf_smem_bytes(stages);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return POT_ERR_CUDA;
+        return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (__half*)Y, prefill_error_ptr());
     };
-    if (bits == 2) return run(pot_gemm_prefill_kernel<2>);
-    if (bits == 3) return run(pot_gemm_prefill_kernel<3>);
-    return run(pot_gemm_prefill_kernel<4>);
+    if (deep) {
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4>, 4);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4>, 4);
+        return run(pot_gemm_prefill_kernel<4, 4>, 4);
+    }
+    if (bits == 2) return run(pot_gemm_prefill_kernel<2, 2>, 2);
+    if (bits == 3) return run(pot_gemm_prefill_kernel<3, 2>, 2);
+    return run(pot_gemm_prefill_kernel<4, 2>, 2);
 }
 
 static int* prefill_error_ptr() { return ring_error_ptr(); }

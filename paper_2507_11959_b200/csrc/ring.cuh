@@ -110,6 +110,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
+// same, but polling with the non-blocking test_wait: a waiter that is parked inside try_wait can take on the
+// order of a microsecond to resume, which is too slow for hand-offs that happen every few hundred cycles
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -224,21 +240,22 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     const int gpr = (int)(K / G);
     const int spg = 128 / G;
 
-    // scales (and zero-points) of a step are fetched one step ahead, straight from global memory
+    // scales (and zero-points) of a step are fetched one step ahead, straight from global memory.  The
+    // buffers keep the raw 16-bit loads: any arithmetic on them here would make the warp wait for the load.
     uint32_t sc[2][2][2], zp[2][2][2];
     auto load_scales = [&](int64_t rb, int c, int buf) {
         const int64_t cb = 4 * (int64_t)c + tig;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            sc[buf][h][0] = sc[buf][h][1] = 0x3C003C00u;
+            sc[buf][h][0] = sc[buf][h][1] = 0x3C00u;
             zp[buf][h][0] = zp[buf][h][1] = 0u;
             if (cb < ncb) {
                 const int64_t so = (rb * 16 + gid + 8 * h) * gpr + cb * spg;
-                sc[buf][h][0] = (uint32_t)__ldg(scales + so) * 0x10001u;
-                sc[buf][h][1] = (uint32_t)__ldg(scales + so + spg - 1) * 0x10001u;
+                sc[buf][h][0] = (uint32_t)__ldg(scales + so);
+                sc[buf][h][1] = (uint32_t)__ldg(scales + so + spg - 1);
                 if constexpr (UNIFORM) {
-                    zp[buf][h][0] = (uint32_t)__ldg(zeros + so) * 0x10001u;
-                    zp[buf][h][1] = (uint32_t)__ldg(zeros + so + spg - 1) * 0x10001u;
+                    zp[buf][h][0] = (uint32_t)__ldg(zeros + so);
+                    zp[buf][h][1] = (uint32_t)__ldg(zeros + so + spg - 1);
                 }
             }
         }
@@ -349,11 +366,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                     for (int h = 0; h < 2; ++h) {
                         uint32_t w2[16];
                         if constexpr (!UNIFORM) {
-                            potl::pot_decode32<BITS>(rec[h], T, sc[buf][h][T >> 1], w2);
+                            potl::pot_decode32<BITS>(rec[h], T, sc[buf][h][T >> 1] * 0x10001u, w2);
                         } else {
                             potl::UintParams pr;
-                            pr.s2 = potl::bits_h2(sc[buf][h][T >> 1]);
-                            pr.z = potl::bits_h2(zp[buf][h][T >> 1]);
+                            pr.s2 = potl::bits_h2(sc[buf][h][T >> 1] * 0x10001u);
+                            pr.z = potl::bits_h2(zp[buf][h][T >> 1] * 0x10001u);
                             potl::uint_decode32<BITS>(rec[h], T, pr, w2);
                         }
 #pragma unroll
@@ -368,8 +385,8 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
 #pragma unroll
             for (int T = 0; T < 4; ++T) {
                 uint32_t w0[16], w1[16];
-                potl::pot_decode32<BITS>(rec[0], T, sc[buf][0][T >> 1], w0);
-                potl::pot_decode32<BITS>(rec[1], T, sc[buf][1][T >> 1], w1);
+                potl::pot_decode32<BITS>(rec[0], T, sc[buf][0][T >> 1] * 0x10001u, w0);
+                potl::pot_decode32<BITS>(rec[1], T, sc[buf][1][T >> 1] * 0x10001u, w1);
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     uint32_t xw[16];
