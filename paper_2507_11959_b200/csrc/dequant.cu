@@ -23,22 +23,35 @@ __device__ __forceinline__ void spread_pairs(uint32_t v, uint32_t (&out)[4]) {
     }
 }
 
+// Piece c = 8 codes = 8*BITS bits starting at bit 8*BITS*c of the stream.  The pieces of one thread are
+// DQ_THREADS apart, i.e. a whole number of words (64*BITS), so word offset and bit phase are computed once.
+template <int BITS>
+__device__ __forceinline__ uint32_t read_piece(const uint32_t* __restrict__ w0, int sh) {
+    const uint32_t lo = __ldg(w0);
+    const uint32_t hi = (sh + 8 * BITS > 32) ? __ldg(w0 + 1) : 0u;
+    const uint32_t v = __funnelshift_r(lo, hi, sh);
+    return (8 * BITS == 32) ? v : (v & ((1u << (8 * BITS % 32)) - 1u));
+}
+
 // PoT: FP16 (EBIT = 10) or BF16 (EBIT = 7) output.
 template <int BITS, int EBIT>
 __global__ void __launch_bounds__(DQ_THREADS) pot_dequant_kernel(const uint32_t* __restrict__ packed,
                                                                  const uint16_t* __restrict__ scales, int64_t n_pieces,
-                                                                 int pieces_per_group, uint4* __restrict__ out) {
+                                                                 int ppg_shift, uint4* __restrict__ out) {
     constexpr uint32_t QM2 = (uint32_t)qmax_of(BITS) * 0x10001u;   // exponent mask, both halves
     constexpr uint32_t SM2 = (1u << (BITS - 1)) * 0x10001u;        // sign mask, both halves
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
+    const int64_t bit0 = base * (8 * BITS);
+    const uint32_t* w0 = packed + (bit0 >> 5);
+    const int sh = (int)(bit0 & 31);
     uint32_t v[DQ_UNROLL];
     uint32_t sc[DQ_UNROLL];
 #pragma unroll
     for (int u = 0; u < DQ_UNROLL; ++u) {
         const int64_t c = base + (int64_t)u * DQ_THREADS;
         if (c < n_pieces) {
-            v[u] = read_bits(packed, c * (8 * BITS), 8 * BITS);
-            sc[u] = __ldg(scales + c / pieces_per_group);
+            v[u] = read_piece<BITS>(w0 + u * (DQ_THREADS * BITS / 4), sh);
+            sc[u] = __ldg(scales + (c >> ppg_shift));
         }
     }
 #pragma unroll
@@ -57,8 +70,9 @@ __global__ void __launch_bounds__(DQ_THREADS) pot_dequant_kernel(const uint32_t*
         for (int j = 0; j < 4; ++j) {
             // stage 1 (bit manipulation): exponent by AND mask, sign moved up, OR;
             // stage 2 (fixed-point add): align with the exponent field and add to the scale's bits.
-            const uint32_t signed_exp = ((pr[j] & QM2) << EBIT) | ((pr[j] & SM2) << (16 - BITS));
-            o[j] = sc2 + signed_exp;
+            // (the power-of-two multiplies are the alignment shifts, fused with the adds into IMADs)
+            const uint32_t e = (pr[j] & QM2) * (1u << EBIT) + sc2;
+            o[j] = (pr[j] & SM2) * (1u << (16 - BITS)) + e;
         }
         out[c] = make_uint4(o[0], o[1], o[2], o[3]);
     }
@@ -70,18 +84,21 @@ template <int BITS>
 __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_fast_kernel(const uint32_t* __restrict__ packed,
                                                                        const uint16_t* __restrict__ scales,
                                                                        const uint16_t* __restrict__ zeros,
-                                                                       int64_t n_pieces, int pieces_per_group,
+                                                                       int64_t n_pieces, int ppg_shift,
                                                                        uint4* __restrict__ out) {
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
+    const int64_t bit0 = base * (8 * BITS);
+    const uint32_t* w0 = packed + (bit0 >> 5);
+    const int sh = (int)(bit0 & 31);
     uint32_t v[DQ_UNROLL];
     uint32_t sc[DQ_UNROLL], zp[DQ_UNROLL];
 #pragma unroll
     for (int u = 0; u < DQ_UNROLL; ++u) {
         const int64_t c = base + (int64_t)u * DQ_THREADS;
         if (c < n_pieces) {
-            v[u] = read_bits(packed, c * (8 * BITS), 8 * BITS);
-            sc[u] = __ldg(scales + c / pieces_per_group);
-            zp[u] = __ldg(zeros + c / pieces_per_group);
+            v[u] = read_piece<BITS>(w0 + u * (DQ_THREADS * BITS / 4), sh);
+            sc[u] = __ldg(scales + (c >> ppg_shift));
+            zp[u] = __ldg(zeros + (c >> ppg_shift));
         }
     }
 #pragma unroll
@@ -109,7 +126,7 @@ template <int BITS>
 __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_naive_kernel(const uint32_t* __restrict__ packed,
                                                                         const uint16_t* __restrict__ scales,
                                                                         const uint16_t* __restrict__ zeros,
-                                                                        int64_t n_pieces, int pieces_per_group,
+                                                                        int64_t n_pieces, int ppg_shift,
                                                                         uint4* __restrict__ out) {
     constexpr uint32_t CM = (1u << BITS) - 1u;
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
@@ -118,8 +135,8 @@ __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_naive_kernel(const ui
         const int64_t c = base + (int64_t)u * DQ_THREADS;
         if (c >= n_pieces) continue;
         const uint32_t v = read_bits(packed, c * (8 * BITS), 8 * BITS);
-        const float s = __half2float(__ushort_as_half(__ldg(scales + c / pieces_per_group)));
-        const float z = __half2float(__ushort_as_half(__ldg(zeros + c / pieces_per_group)));
+        const float s = __half2float(__ushort_as_half(__ldg(scales + (c >> ppg_shift))));
+        const float z = __half2float(__ushort_as_half(__ldg(zeros + (c >> ppg_shift))));
         uint32_t o[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -149,7 +166,7 @@ extern "C" pot_status_t pot_dequant(const void* packed, const void* scales, int6
     auto* P = (const uint32_t*)packed;
     auto* S = (const uint16_t*)scales;
     auto* O = (uint4*)W_out;
-    const int ppg = group / 8;
+    const int ppg = group == 64 ? 3 : 4;  // log2(pieces per group): a 64-bit division per piece would dominate the kernel
 #define POT_DQ(B)                                                                                     \
     if (out_dtype == POT_F16) pot_dequant_kernel<B, 10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O); \
     else pot_dequant_kernel<B, 7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
@@ -172,7 +189,7 @@ extern "C" pot_status_t uint_dequant(const void* packed, const void* scales, con
     auto* S = (const uint16_t*)scales;
     auto* Z = (const uint16_t*)zeros;
     auto* O = (uint4*)W_out;
-    const int ppg = group / 8;
+    const int ppg = group == 64 ? 3 : 4;  // log2(pieces per group): a 64-bit division per piece would dominate the kernel
 #define UINT_DQ(B)                                                                                              \
     if (kernel == UINT_KERNEL_FAST) uint_dequant_fast_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O); \
     else uint_dequant_naive_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
