@@ -89,13 +89,12 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * PF_STAGE_BYTES);
-    // bars: fullA[S], fullB[S], empty[S], accum, then the tensor-memory base address
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * PF_STAGES + 1);
+    // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PF_STAGES + 1);
     const uint32_t bar0 = smem_u32(bars);
-    auto fullA = [&](int s) { return bar0 + 8u * s; };
-    auto fullB = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
-    auto empty = [&](int s) { return bar0 + 8u * (2 * PF_STAGES + s); };
-    const uint32_t accum = bar0 + 8u * (3 * PF_STAGES);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
+    const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.x * (PF_BM * PF_MT), n0 = (int64_t)blockIdx.y * PF_BN;
@@ -104,8 +103,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
-            mbar_init(fullA(s), 1);
-            mbar_init(fullB(s), PF_PRODUCERS);   // one arrival per producer warp
+            mbar_init(full(s), 1 + PF_PRODUCERS / 2);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
             mbar_init(empty(s), 1);
         }
         mbar_init(accum, 1);
@@ -130,22 +128,27 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
                 }
-                mbar_expect_tx(fullA(s), PF_MT * PF_ATOM_BYTES);
+                mbar_expect_tx(full(s), PF_MT * PF_ATOM_BYTES);
                 const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
 #pragma unroll
                 for (int mt = 0; mt < PF_MT; ++mt)
-                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, kb * PF_BK, (int)m0 + mt * PF_BM, fullA(s));
+                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, kb * PF_BK, (int)m0 + mt * PF_BM, full(s));
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------
         if (lane == 0) {
+            // A barrier test costs a few hundred cycles even when the phase is long complete, so the test for
+            // stage kb+1 is put in flight before the MMAs of stage kb are issued and only examined afterwards.
+            uint32_t ready = mbar_test(full(0), 0);
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % PF_STAGES;
                 const uint32_t ph = (uint32_t)((kb / PF_STAGES) & 1);
-                if (!mbar_wait(fullA(s), ph) || !mbar_wait(fullB(s), ph)) {
+                if (!ready && !mbar_wait(full(s), ph)) {
                     if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
                 }
+                ready = 0;
+                if (kb + 1 < nkb) ready = mbar_test(full((kb + 1) % PF_STAGES), (uint32_t)(((kb + 1) / PF_STAGES) & 1));
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES), b = a + PF_MT * PF_ATOM_BYTES;
 #pragma unroll
@@ -160,23 +163,25 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         }
     } else {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
-        const int pt = threadIdx.x - 64;            // 0..255
-        const int row = pt & 127, qsel = pt >> 7;   // weight row inside the tile; which 32 of the stage's 64 columns
+        // Two groups of four warps take alternate stages: a stage visit costs a warp a fixed ~1000 cycles of
+        // hand-off latency (barrier test, proxy fence, arrive), so more stages must be in preparation at once.
+        // Stage kb covers columns 64*kb .. 64*kb+63, i.e. half (kb & 1) of column block kb / 2; group g owns the
+        // stages with kb & 1 == g, hence always the same half of the records.  Thread = one weight row.
+        const int pt = threadIdx.x - 64;          // 0..255
+        const int grp = pt >> 7, row = pt & 127;
         const int64_t n = n0 + row;
         const bool row_ok = n < N;
         const int64_t rb = n >> 4;
         const int r = (int)(n & 15);
         const int gpr = (int)(K / G), spg = 128 / G;
+        const int w_lo = grp * (NW / 2), w_hi = w_lo + NW / 2 - 1;   // words of this group's half record
 
-        // stage kb covers columns 64*kb .. 64*kb+63 = quarter-records T = 2*(kb&1) + qsel of column block kb/2
-        // The packed codes are prefetched PF_DEPTH - 1 stages ahead (a stage lasts less than a memory latency).
-        constexpr int PF_DEPTH = 4;
+        // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.
+        constexpr int PF_DEPTH = (BITS == 4 && PF_STAGES == 2) ? 3 : 4;  // 4-bit records at 96 registers: one buffer fewer
         uint32_t rec[PF_DEPTH][NW];
         uint32_t sc2[PF_DEPTH];
         auto load = [&](int kb, int buf) {
             if (row_ok) {
-                const int T = 2 * (kb & 1) + qsel;
-                const int w_lo = T * (NW / 4), w_hi = w_lo + NW / 4 - 1;   // the quarter record's words
                 const uint4* unit = packed + (rb * ncb + (kb >> 1)) * (16 * BITS);
 #pragma unroll
                 for (int t = 0; t < BITS; ++t) {
@@ -185,19 +190,21 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                         rec[buf][4 * t + 0] = q.x; rec[buf][4 * t + 1] = q.y; rec[buf][4 * t + 2] = q.z; rec[buf][4 * t + 3] = q.w;
                     }
                 }
-                const int64_t so = n * gpr + (int64_t)(kb >> 1) * spg + (spg == 2 ? (kb & 1) : 0);
+                const int64_t so = n * gpr + (int64_t)(kb >> 1) * spg + (spg == 2 ? grp : 0);
                 sc2[buf] = (uint32_t)__ldg(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
+        const int nmine = (nkb - grp + 1) / 2;   // stages kb = grp, grp + 2, ...
 #pragma unroll
         for (int p = 0; p < PF_DEPTH - 1; ++p)
-            if (p < nkb) load(p, p);
-        for (int kb4 = 0; kb4 < nkb; kb4 += PF_DEPTH) {
+            if (p < nmine) load(2 * p + grp, p);
+        for (int i4 = 0; i4 < nmine; i4 += PF_DEPTH) {
 #pragma unroll
             for (int buf = 0; buf < PF_DEPTH; ++buf) {
-                const int kb = kb4 + buf;
-                if (kb >= nkb) break;
-                if (kb + PF_DEPTH - 1 < nkb) load(kb + PF_DEPTH - 1, (buf + PF_DEPTH - 1) % PF_DEPTH);
+                const int i = i4 + buf;
+                if (i >= nmine) break;
+                const int kb = 2 * i + grp;
+                if (i + PF_DEPTH - 1 < nmine) load(kb + 2 * (PF_DEPTH - 1), (buf + PF_DEPTH - 1) % PF_DEPTH);
                 const int s = kb % PF_STAGES;
                 if (kb >= PF_STAGES) {  // one lane polls for the whole warp: the warp is about to WRITE the stage
                     if (lane == 0 && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
@@ -205,26 +212,28 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
                     __syncwarp();
                 }
-                uint32_t w2[16];
-                if (row_ok) {
-                    // buf has the parity of kb, so the quarter index 2*(kb&1) + qsel is static in each branch
-                    const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
-                    if (qsel == 0) potl::pot_decode32<BITS>(rec[buf], 2 * (buf & 1), s2, w2);
-                    else potl::pot_decode32<BITS>(rec[buf], 2 * (buf & 1) + 1, s2, w2);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) w2[i] = 0u;
-                }
                 unsigned char* brow = smem + (size_t)s * PF_STAGE_BYTES + PF_MT * PF_ATOM_BYTES + row * 128;
+                const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {  // 4 chunks of 8 halves; chunk index inside the 128-byte row
-                    const int chunk = 4 * qsel + c;
-                    *reinterpret_cast<uint4*>(brow + ((chunk ^ (row & 7)) << 4)) =
-                        make_uint4(w2[4 * c], w2[4 * c + 1], w2[4 * c + 2], w2[4 * c + 3]);
+                for (int T2 = 0; T2 < 2; ++T2) {
+                    uint32_t w2[16];
+                    if (row_ok) {
+                        if (grp == 0) potl::pot_decode32<BITS>(rec[buf], T2, s2, w2);
+                        else potl::pot_decode32<BITS>(rec[buf], 2 + T2, s2, w2);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) w2[q] = 0u;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {  // 4 chunks of 8 halves; chunk index inside the 128-byte row
+                        const int chunk = 4 * T2 + c;
+                        *reinterpret_cast<uint4*>(brow + ((chunk ^ (row & 7)) << 4)) =
+                            make_uint4(w2[4 * c], w2[4 * c + 1], w2[4 * c + 2], w2[4 * c + 3]);
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(fullB(s));
+                if (lane == 0) mbar_arrive(full(s));
             }
         }
         // ---------------- epilogue: tensor memory -> registers -> FP16 -> Y --------------------------

@@ -110,6 +110,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
+// one non-blocking test (1 = the phase with this parity has completed)
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done;
+}
 // same, but polling with the non-blocking test_wait: a waiter that is parked inside try_wait can take on the
 // order of a microsecond to resume, which is too slow for hand-offs that happen every few hundred cycles
 __device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
