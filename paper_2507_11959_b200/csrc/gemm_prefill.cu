@@ -84,7 +84,6 @@ __global__ void __launch_bounds__(PF_THREADS, PF_STAGES == 2 ? 2 : 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
                         __half* __restrict__ Y, int* __restrict__ err) {
-    constexpr int NW = 4 * BITS;
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -174,21 +173,18 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         const int64_t rb = n >> 4;
         const int r = (int)(n & 15);
         const int gpr = (int)(K / G), spg = 128 / G;
-        const int w_lo = grp * (NW / 2), w_hi = w_lo + NW / 2 - 1;   // words of this group's half record
-
-        // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.
+        // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.  Every 16-byte plane of the
+        // row holds one word of each quarter; the group needs quarters 2*grp and 2*grp + 1: 8 bytes per plane.
         constexpr int PF_DEPTH = (BITS == 4 && PF_STAGES == 2) ? 3 : 4;  // 4-bit records at 96 registers: one buffer fewer
-        uint32_t rec[PF_DEPTH][NW];
+        uint32_t rec[PF_DEPTH][2 * BITS];
         uint32_t sc2[PF_DEPTH];
         auto load = [&](int kb, int buf) {
             if (row_ok) {
-                const uint4* unit = packed + (rb * ncb + (kb >> 1)) * (16 * BITS);
+                const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + (kb >> 1)) * (16 * BITS));
 #pragma unroll
                 for (int t = 0; t < BITS; ++t) {
-                    if (t >= (w_lo >> 2) && t <= (w_hi >> 2)) {
-                        const uint4 q = __ldg(unit + t * 16 + r);
-                        rec[buf][4 * t + 0] = q.x; rec[buf][4 * t + 1] = q.y; rec[buf][4 * t + 2] = q.z; rec[buf][4 * t + 3] = q.w;
-                    }
+                    const uint2 q = __ldg(unit + (t * 16 + r) * 2 + grp);
+                    rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
                 }
                 const int64_t so = n * gpr + (int64_t)(kb >> 1) * spg + (spg == 2 ? grp : 0);
                 sc2[buf] = (uint32_t)__ldg(scales + so);  // raw bits: any arithmetic here would stall on the load
@@ -218,8 +214,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 for (int T2 = 0; T2 < 2; ++T2) {
                     uint32_t w2[16];
                     if (row_ok) {
-                        if (grp == 0) potl::pot_decode32<BITS>(rec[buf], T2, s2, w2);
-                        else potl::pot_decode32<BITS>(rec[buf], 2 + T2, s2, w2);
+                        potl::pot_decode32<BITS, 2>(rec[buf], T2, s2, w2);
                     } else {
 #pragma unroll
                         for (int q = 0; q < 16; ++q) w2[q] = 0u;

@@ -2,31 +2,34 @@
 //
 // One "record" = the 128 codes of one row inside one 128-column block = 4n 32-bit words.
 // The map below says where bit b of code q (0 <= q < 128) lives: (word index, bit position).
-// Codes 2P and 2P+1 ("pair" P) always sit 16 bits apart in one word, so that one AND mask
-// and one multiply-add (shift left + add the scale's bit pattern, Sec. 4.2 of the paper)
-// produce both halves of a half2.  The PoT maps additionally put the sign bit where the same
-// shift moves it to bit 15 (n = 2), or in a position of its own (n = 3, 4).
 //
-//  PoT n = 2 : word w = q/16 holds codes 16w..16w+15; pair p = (q%16)/2, half h = q%2.
-//              The word is a ring of 32 positions; a code anchored at even position a has
-//              its exponent bit at a and its sign at a+5 (mod 32):
-//                p <= 5 : anchor 2p + 16h           (decoded straight from the word)
-//                p == 6 : anchor 28 (h=0), 12 (h=1) (decoded after rotating the word left by 8)
-//                p == 7 : anchor 30 (h=0), 14 (h=1)
-//  PoT n = 3 : the record is four "triples" of three words; triple T = q/32 holds pairs
-//              P = (q%32)/2 = 0..15.  Pair P < 15 lives in word 3T + P/5 as slot d = P%5:
-//                d < 4 : exponent at bits 3d, 3d+1 and sign at 3d+5 (+16h) -- the sign sits five
-//                        positions above the exponent's low bit, so ONE mask and ONE shift-add
-//                        place both (these are 12 of every 16 pairs);
-//                d = 4 : exponent at bits 12,13 and sign already at bit 15 (+16h);
-//              pair 15 is spread over bit 2 (+16h) of the three words: exponent bit 0 in word
-//              3T, exponent bit 1 in word 3T+1, sign in word 3T+2.
-//              (The uniform twin keeps the plain plane map: words 0..7 hold the low two bits as
-//              fields 2p + 16h, words 8..11 the high bit at (q%32)/2 + 16h.)
-//  PoT n = 4 : word w = q/8 holds codes 8w..8w+7; pair p = (q%8)/2; exponent at bits
-//              3p + 16h + {0,1,2}, sign at bit 12 + p + 16h.
-//  uniform   : the n-bit integer code as a field: n = 2 at 2p + 16h (p < 8), n = 4 at
-//              4p + 16h (p < 4), n = 3 as for PoT n = 3 (low two bits / high bit planes).
+// PoT codes ("byte-lane" map).  Quarter T = q / 32 of the record owns the n words 4k + T
+// (k = 0..n-1; word k of every quarter sits in 16-byte plane k of the row).  A quarter decodes
+// into eight "decoded words" i = 0..7 of four byte lanes each; byte lane l of decoded word i is
+// column 32T + 4i + perm[l], perm = {0, 2, 1, 3} -- so lanes (0, 2) and (1, 3), which sit 16
+// bits apart, are pairs of ADJACENT columns.  Inside a byte lane the code is stored in the shape
+// of an 8-bit float with five exponent bits: exponent bits from bit 2 upwards, sign at bit 7
+// (five above the exponent's low bit), after a rotation of the word:
+//   * as FP8 operand : (rot(w) & mask) | 0x40..  is the byte pattern of +-2^(E+1) -- one
+//                      logic operation per four weights, consumed by the FP8 tensor-core MMA;
+//   * as FP16 pair   : (rot(w) & mask16) * 2^8 + scale  (lanes 0, 2)  and
+//                      (rot(w) & mask16 << 8) + scale   (lanes 1, 3)  -- the mask / shift /
+//                      integer add into the scale's bit pattern of Sec. 4.2 of the paper.
+// A "plane" (word k, anchor a) stores exponent bit e of lane l at bit (8l + a + e) mod 32 and the
+// sign at (8l + a + 5) mod 32; rotating the word right by a - 2 brings it into place.
+//  PoT n = 2 : words k = 0, 1; anchors 0, 2, 4, 6; decoded word i = 4k + a/2.
+//  PoT n = 3 : words k = 0, 1, 2 with anchors {1,3}, {4,6}, {5,7}: decoded word i = 2k + (0|1).
+//              Each word keeps two spare bits per byte lane ({5,7}, {0,2}, {1,3}); they hold
+//              decoded word 6 = {sign: word 0 bit 7, E0: word 1 bit 2, E1: word 2 bit 3} (all in
+//              place) and decoded word 7 = {sign: word 0 bit 5, E0: word 1 bit 0, E1: word 2
+//              bit 1} (in place after a shift left by 2).
+//  PoT n = 4 : words k = 0..3, decoded word i = 2k + (0|1): plane 0 in place (E at 2,3,4, sign
+//              at 7), plane 1 = {E0, E1 at 0, 1; sign at 5} (rotate left 2) + {E2 at 6} (rotate
+//              right 2).
+// Uniform codes keep the n-bit integer as one field, pairs 16 bits apart:
+//  n = 2 at 2p + 16h (p < 8, word q/16), n = 4 at 4p + 16h (p < 4, word q/8), n = 3 as two
+//  planes: words 0..7 hold the low two bits as fields 2p + 16h, words 8..11 the high bit at
+//  (q%32)/2 + 16h  (pair p = (q % codes-per-word) / 2, half h = q % 2).
 #pragma once
 #include <cstdint>
 
@@ -39,23 +42,44 @@ struct BitPos {
     int bit;
 };
 
-// where bit b of code q is stored inside the record
+// where bit b of code q is stored inside the record (b < n-1: exponent bits, b = n-1: sign, for PoT)
 __host__ __device__ inline BitPos record_bit(int bits, int kind, int q, int b) {
     BitPos r;
+    if (kind == KIND_POT) {
+        const int T = q >> 5, c = q & 31;
+        const int i = c >> 2;                                       // decoded word
+        const int l = ((c & 1) << 1) | ((c >> 1) & 1);              // byte lane: perm is its own inverse
+        const bool sign = (b == bits - 1);
+        int k, pos;
+        if (bits == 2) {
+            k = i >> 2;
+            pos = 8 * l + 2 * (i & 3) + (sign ? 5 : 0);
+        } else if (bits == 4) {
+            k = i >> 1;
+            if ((i & 1) == 0) pos = 8 * l + (sign ? 7 : 2 + b);
+            else pos = 8 * l + (sign ? 5 : (b == 2 ? 6 : b));
+        } else {
+            if (i < 6) {
+                k = i >> 1;
+                const int a = (k == 0 ? 1 : (k == 1 ? 4 : 5)) + 2 * (i & 1);
+                pos = 8 * l + a + (sign ? 5 : b);
+            } else if (i == 6) {
+                k = sign ? 0 : 1 + b;
+                pos = 8 * l + (sign ? 7 : 2 + b);
+            } else {
+                k = sign ? 0 : 1 + b;
+                pos = 8 * l + (sign ? 5 : b);
+            }
+        }
+        r.word = 4 * k + T;
+        r.bit = pos & 31;
+        return r;
+    }
     const int h = q & 1;
     if (bits == 2) {
         r.word = q >> 4;
-        const int p = (q & 15) >> 1;
-        if (kind == KIND_UINT) {
-            r.bit = 2 * p + 16 * h + b;
-        } else {
-            int anchor;
-            if (p <= 5) anchor = 2 * p + 16 * h;
-            else if (p == 6) anchor = h ? 12 : 28;
-            else anchor = h ? 14 : 30;
-            r.bit = (b == 0) ? anchor : ((anchor + 5) & 31);
-        }
-    } else if (bits == 3 && kind == KIND_UINT) {
+        r.bit = 2 * ((q & 15) >> 1) + 16 * h + b;
+    } else if (bits == 3) {
         if (b < 2) {
             r.word = q >> 4;
             r.bit = 2 * ((q & 15) >> 1) + 16 * h + b;
@@ -63,119 +87,106 @@ __host__ __device__ inline BitPos record_bit(int bits, int kind, int q, int b) {
             r.word = 8 + (q >> 5);
             r.bit = ((q & 31) >> 1) + 16 * h;
         }
-    } else if (bits == 3) {
-        const int T = q >> 5, P = (q & 31) >> 1;
-        if (P < 15) {
-            const int d = P % 5;
-            r.word = 3 * T + P / 5;
-            if (d < 4) r.bit = 3 * d + 16 * h + (b < 2 ? b : 5);
-            else r.bit = 16 * h + (b < 2 ? 12 + b : 15);
-        } else {
-            r.word = 3 * T + b;
-            r.bit = 2 + 16 * h;
-        }
     } else {
         r.word = q >> 3;
-        const int p = (q & 7) >> 1;
-        if (kind == KIND_UINT) r.bit = 4 * p + 16 * h + b;
-        else r.bit = (b < 3) ? (3 * p + 16 * h + b) : (12 + p + 16 * h);
+        r.bit = 4 * ((q & 7) >> 1) + 16 * h + b;
     }
     return r;
 }
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------------------
-// Register decoders.  `sc2` is the group scale's FP16 bit pattern replicated in both halves.
-// Each returns the bit pattern of half2{ w~[2P], w~[2P+1] } for pair P of the record.
-// mad(t, c, s) = t * c + s is one IMAD: the multiply by a power of two is the shift that aligns
-// the exponent with FP16 bit 10 and the sign with bit 15, the add is the "fixed-point integer
-// addition" into the scale (Sec. 4.2).
+// Register decoders for the PoT byte-lane map.
+// rotated_words<BITS>(w, d): the quarter's n words -> its eight decoded words, every code rotated
+// into place (exponent from bit 2, sign at bit 7 of its byte lane) but NOT yet masked; decoded
+// word 7 of n = 3 is the exception: its bits sit two positions low (flagged by LOW7).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t mad(uint32_t t, uint32_t c, uint32_t s) { return t * c + s; }
+__device__ __forceinline__ uint32_t rotr(uint32_t v, int s) { return __funnelshift_r(v, v, s); }
 __device__ __forceinline__ uint32_t rotl(uint32_t v, int s) { return __funnelshift_l(v, v, s); }
+// bitwise select: mask bits from a, the others from b (one LOP3)
+__device__ __forceinline__ uint32_t sel(uint32_t a, uint32_t b, uint32_t mask) { return (a & mask) | (b & ~mask); }
 
 template <int BITS>
-struct PotDecoder;
-
-// n = 2 : 16 codes (8 pairs) per word, 2 operations per pair + one rotate per word.
+struct PotLanes;
 template <>
-struct PotDecoder<2> {
-    static constexpr int WORDS = 8;
-    static constexpr int PAIRS_PER_WORD = 8;
-    // out[8]: pairs 8w .. 8w+7
-    static __device__ __forceinline__ void word(uint32_t w, uint32_t sc2, uint32_t (&out)[8]) {
+struct PotLanes<2> {
+    static constexpr uint32_t MASK = 0x84848484u;
+    static constexpr bool LOW7 = false;
+    static __device__ __forceinline__ void rotate(const uint32_t (&w)[2], uint32_t (&d)[8]) {
 #pragma unroll
-        for (int p = 0; p < 6; ++p) out[p] = mad(w & (0x00210021u << (2 * p)), 1u << (10 - 2 * p), sc2);
-        const uint32_t r = rotl(w, 8);
-        out[6] = mad(r & 0x02100210u, 64u, sc2);
-        out[7] = mad(r & 0x08400840u, 16u, sc2);
+        for (int k = 0; k < 2; ++k) {
+            d[4 * k + 0] = rotl(w[k], 2);
+            d[4 * k + 1] = w[k];
+            d[4 * k + 2] = rotr(w[k], 2);
+            d[4 * k + 3] = rotr(w[k], 4);
+        }
     }
 };
-
-// n = 4 : 8 codes (4 pairs) per word; exponent and sign are placed by two multiply-adds.
 template <>
-struct PotDecoder<4> {
-    static constexpr int WORDS = 16;
-    static constexpr int PAIRS_PER_WORD = 4;
-    static __device__ __forceinline__ void word(uint32_t w, uint32_t sc2, uint32_t (&out)[4]) {
+struct PotLanes<3> {
+    static constexpr uint32_t MASK = 0x8C8C8C8Cu;
+    static constexpr bool LOW7 = true;
+    static __device__ __forceinline__ void rotate(const uint32_t (&w)[3], uint32_t (&d)[8]) {
+        d[0] = rotl(w[0], 1);
+        d[1] = rotr(w[0], 1);
+        d[2] = rotr(w[1], 2);
+        d[3] = rotr(w[1], 4);
+        d[4] = rotr(w[2], 3);
+        d[5] = rotr(w[2], 5);
+        d[6] = sel(sel(w[0], w[1], 0x80808080u), w[2], 0x84848484u);
+        d[7] = sel(sel(w[0], w[1], 0x20202020u), w[2], 0x21212121u);  // two positions low
+    }
+};
+template <>
+struct PotLanes<4> {
+    static constexpr uint32_t MASK = 0x9C9C9C9Cu;
+    static constexpr bool LOW7 = false;
+    static __device__ __forceinline__ void rotate(const uint32_t (&w)[4], uint32_t (&d)[8]) {
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            const uint32_t e = mad(w & (0x00070007u << (3 * p)), 1u << (10 - 3 * p), sc2);
-            if (p == 3) out[p] = e | (w & 0x80008000u);
-            else out[p] = mad(w & (0x10001000u << p), 1u << (3 - p), e);
+        for (int k = 0; k < 4; ++k) {
+            d[2 * k] = w[k];
+            d[2 * k + 1] = sel(rotl(w[k], 2), rotr(w[k], 2), 0x8C8C8C8Cu);
         }
     }
 };
 
-// n = 3 : three words hold 16 pairs (see the map at the top of this file).
-template <>
-struct PotDecoder<3> {
-    static constexpr int WORDS = 12;
-    // out[16]: pairs 16T .. 16T+15 of the record, from words w0, w1, w2 of triple T
-    static __device__ __forceinline__ void triple(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sc2,
-                                                  uint32_t (&out)[16]) {
-        const uint32_t w[3] = {w0, w1, w2};
-#pragma unroll
-        for (int j = 0; j < 3; ++j) {
-#pragma unroll
-            for (int d = 0; d < 4; ++d) out[5 * j + d] = mad(w[j] & (0x00230023u << (3 * d)), 1u << (10 - 3 * d), sc2);
-            // slot 4: exponent at bits 12,13 (two positions too high), sign in place at bit 15
-            const uint32_t e = (__funnelshift_r(w[j], w[j], 2) & 0x0C000C00u) + sc2;
-            out[5 * j + 4] = e | (w[j] & 0x80008000u);
-        }
-        uint32_t y = mad(w0 & 0x00040004u, 1u << 8, sc2);
-        y = mad(w1 & 0x00040004u, 1u << 9, y);
-        out[15] = mad(w2 & 0x00040004u, 1u << 13, y);
-    }
-};
-
-// Decode 32 consecutive codes (16 pairs): quarter T (0..3) of a record held in registers.
+// Quarter -> eight words of four FP8 (five exponent bits, two mantissa bits) bytes: byte lane l of
+// word i is +-2^(E+1) for column 4i + perm[l] of the quarter.  The constant 0x40 per byte sets
+// the exponent field to 16 + E.
 template <int BITS>
-__device__ __forceinline__ void pot_decode32(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]);
-
-template <>
-__device__ __forceinline__ void pot_decode32<2>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
-    uint32_t a[8], b[8];
-    PotDecoder<2>::word(rec[2 * T], sc2, a);
-    PotDecoder<2>::word(rec[2 * T + 1], sc2, b);
+__device__ __forceinline__ void pot_decode32_f8(const uint32_t (&w)[BITS], uint32_t (&dw)[8]) {
+    using L = PotLanes<BITS>;
+    uint32_t d[8];
+    L::rotate(w, d);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        out[i] = a[i];
-        out[8 + i] = b[i];
+        if (L::LOW7 && i == 7) dw[i] = mad(d[i] & (L::MASK >> 2), 4u, 0x40404040u);
+        else dw[i] = (d[i] & L::MASK) | 0x40404040u;
     }
 }
-template <>
-__device__ __forceinline__ void pot_decode32<3>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
-    PotDecoder<3>::triple(rec[3 * T], rec[3 * T + 1], rec[3 * T + 2], sc2, out);
-}
-template <>
-__device__ __forceinline__ void pot_decode32<4>(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
+
+// Decode 32 consecutive codes (16 pairs): quarter T (0..3) of a record held in registers
+// (rec[STRIDE * k + T] = word k of the quarter; STRIDE = 4 for a whole record).  out[p] = bit pattern of half2{ w~[2p], w~[2p+1] }:
+// mask, align with the FP16 exponent / sign (the multiply by a power of two is the shift) and
+// integer-add to the scale's bit pattern `sc2` (both halves) -- Sec. 4.2 of the paper.
+template <int BITS, int STRIDE = 4>
+__device__ __forceinline__ void pot_decode32(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
+    using L = PotLanes<BITS>;
+    constexpr uint32_t MA = L::MASK & 0x00FF00FFu, MB = L::MASK & 0xFF00FF00u;
+    uint32_t w[BITS], d[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint32_t a[4];
-        PotDecoder<4>::word(rec[4 * T + i], sc2, a);
+    for (int k = 0; k < BITS; ++k) w[k] = rec[STRIDE * k + T];
+    L::rotate(w, d);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) out[4 * i + k] = a[k];
+    for (int i = 0; i < 8; ++i) {
+        if (L::LOW7 && i == 7) {
+            out[2 * i] = mad(d[i] & (MA >> 2), 1u << 10, sc2);
+            out[2 * i + 1] = mad(d[i] & (MB >> 2), 1u << 2, sc2);
+        } else {
+            out[2 * i] = mad(d[i] & MA, 1u << 8, sc2);
+            out[2 * i + 1] = (d[i] & MB) + sc2;
+        }
     }
 }
 

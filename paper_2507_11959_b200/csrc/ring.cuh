@@ -31,7 +31,7 @@ constexpr int RG_CONSUMERS = 15;
 constexpr int RG_THREADS = (RG_CONSUMERS + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2 };
+enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3 };
 
 constexpr int RG_Q = 5;  // steps per ring slot (one bulk copy) = warps per consumer group
 constexpr int RG_GROUPS = RG_CONSUMERS / RG_Q;  // slot m is consumed by group m % RG_GROUPS, warp i of it takes step i
@@ -53,13 +53,13 @@ struct RingPlan {
     size_t ws_bytes;
 };
 
-inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok) {
+inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bool wide_ok = true) {
     RingPlan p;
     const int64_t nrb = N / 16, ncb = K / 128;
     p.spr = (int)((ncb + 3) / 4);
     p.total_steps = nrb * p.spr;
     p.grid = (int)(p.total_steps < kSmCount ? p.total_steps : kSmCount);
-    p.x_wide = (tok == 1) && (size_t)K * 4 <= 48 * 1024;
+    p.x_wide = wide_ok && (tok == 1) && (size_t)K * 4 <= 48 * 1024;
     const size_t xb = (size_t)M * (size_t)K * (p.x_wide ? 4 : 2);
     p.x_in_smem = xb <= 64 * 1024;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
@@ -177,7 +177,11 @@ __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// MODE RG_POT_FMA / RG_UINT_FMA: M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
+// MODE RG_POT_FMA / RG_UINT_FMA / RG_POT_MMA1: M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
+// RG_POT_MMA1 is the GEMV on the warp-level tensor-core path: the activation vector fills every column of the
+// MMA's B operand, lane (gid, tig) owns quarter tig of the records of rows gid and gid + 8 -- exactly its share
+// of the A fragment -- and the MMA adds up the four quarters, so there is no cross-lane reduction and the
+// multiply-accumulate costs one instruction per 256 weights instead of one per weight.
 template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = staged packed, 2 = staged wide
 __global__ void __launch_bounds__(RG_THREADS, 1)
 ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
@@ -189,6 +193,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     constexpr bool XWIDE = (XMODE == 2);
     constexpr bool MMA = (MODE == RG_POT_MMA);
     constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
+    constexpr bool MMA1 = (MODE == RG_POT_MMA1);
     constexpr int TOK = MMA ? 8 * MT : 1;
     constexpr int SLOT = rg_slot_bytes(BITS);
     constexpr int UB = rg_unit_bytes(BITS);
@@ -247,15 +252,32 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     }
 
     // -------------------- consumers --------------------------------------------------------------------
-    const int gid = MMA ? (lane >> 2) : (lane & 7);
-    const int tig = MMA ? (lane & 3) : (lane >> 3);
+    const int gid = (MMA || MMA1) ? (lane >> 2) : (lane & 7);
+    const int tig = (MMA || MMA1) ? (lane & 3) : (lane >> 3);
     const int gpr = (int)(K / G);
     const int spg = 128 / G;
 
     // scales (and zero-points) of a step are fetched one step ahead, straight from global memory.  The
     // buffers keep the raw 16-bit loads: any arithmetic on them here would make the warp wait for the load.
+    // RG_POT_MMA1: the scale of this lane's quarter, for both rows and the four units of a step
+    uint32_t sc1[2][MMA1 ? 8 : 1];
+    auto load_scales_mma1 = [&](int64_t rb, int c, int buf) {
+        // one 64-bit address per step; the eight loads use constant offsets from it
+        const uint16_t* s0 = scales + (rb * 16 + gid) * gpr + (int64_t)c * (4 * spg) + (spg == 2 ? (tig >> 1) : 0);
+        const int64_t up = 8 * (int64_t)gpr;
+        const int nu = (int)(ncb - 4 * (int64_t)c);  // units of this step (>= 4 except at the ragged end of a row)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint32_t v = 0x3C00u;
+                if (u < nu) v = (uint32_t)__ldg(s0 + (h ? up : 0) + (spg == 2 ? 2 * u : u));
+                sc1[buf][h * 4 + u] = v;
+            }
+    };
     uint32_t sc[2][2][2], zp[2][2][2];
     auto load_scales = [&](int64_t rb, int c, int buf) {
+        if constexpr (MMA1) { load_scales_mma1(rb, c, buf); return; }
         const int64_t cb = 4 * (int64_t)c + tig;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -294,6 +316,10 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             if constexpr (XWIDE) {
                 dst[2 * i] = make_uint4(v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16);
                 dst[2 * i + 1] = make_uint4(v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16);
+            } else if constexpr (MMA1) {
+                // chunk (quarter t, part j) of a unit goes to position j * 4 + t: the four lanes tig = 0..3 then
+                // read 64 contiguous bytes
+                dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v;
             } else {
                 dst[i] = v;
             }
@@ -327,6 +353,54 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         if (!mbar_wait(smem_u32(&bars[slot]), phase)) {
             if (err && lane == 0) atomicCAS(err, 0, 2 | (m << 8) | (warp << 16) | (j << 24));
         }
+        float r0 = 0.f, r1 = 0.f;  // RG_POT_MMA1: the sums of rows gid and gid + 8
+        if constexpr (MMA1) {
+            // units between the slot's first step (wig steps back) and this one, without divisions
+            int64_t rb_s = rb;
+            int c_s = c - wig;
+            while (c_s < 0) { c_s += spr; --rb_s; }
+            const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - (rb_s * ncb + 4 * (int64_t)c_s);
+            // plane k of a unit holds word k of every (row, quarter): this lane's word sits at byte 4 * lane
+            const unsigned char* ubase = ring + (size_t)slot * SLOT + uoff * UB + lane * 4;
+            float acc1[2][4];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t cbu = 4 * (int64_t)c + u;
+                if (cbu < ncb) {  // the same for the whole warp
+                    uint32_t w[2][BITS];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int k = 0; k < BITS; ++k)
+                            w[h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
+                    uint32_t xq[16];  // the 32 activations of quarter tig: the B fragments of eight MMAs
+                    {
+                        const uint4* xp = (XSMEM ? xs : reinterpret_cast<const uint4*>(X)) + cbu * 16 + (XSMEM ? tig : tig * 4);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 v = XSMEM ? xp[4 * i] : __ldg(xp + i);
+                            xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
+                        }
+                    }
+                    uint32_t lo[16], hi[16];
+                    potl::pot_decode32<BITS, 1>(w[0], 0, sc1[buf][u] * 0x10001u, lo);
+                    potl::pot_decode32<BITS, 1>(w[1], 0, sc1[buf][4 + u] * 0x10001u, hi);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)  // two accumulators: half the length of the dependent chain
+                        rg_mma(acc1[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
+            r0 = acc1[0][0] + acc1[1][0];   // every column of the product holds the same sums
+            r1 = acc1[0][2] + acc1[1][2];
+        }
+        float acc[MMA ? 4 * MT : 4];
+        if constexpr (!MMA1) {
         uint32_t rec[2][NW];
         {
             // records are fetched with lane (column block, row) = (lane / 8, lane % 8): 8 lanes read 128
@@ -359,7 +433,6 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
 
-        float acc[MMA ? 4 * MT : 4];
 #pragma unroll
         for (int i = 0; i < (MMA ? 4 * MT : 4); ++i) acc[i] = 0.f;
         if (!MMA) {
@@ -418,6 +491,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             }
         }
 
+        }
         // ---- deliver the step's partial sums -----------------------------------------------------------
         // spr == 1: the step is the whole row block, write Y.  Otherwise the 16*TOK sums go to a slot:
         // in shared memory when every step of the row block belongs to this CTA (the common case),
@@ -429,9 +503,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                             : (local ? cmb + (size_t)(rb_g0 - g_begin + c) * (16 * TOK)
                                      : partial + (rb_g0 + c) * (16 * TOK));
         if (!MMA) {
-            float r0 = acc[0] + acc[1], r1 = acc[2] + acc[3];
-            r0 += __shfl_xor_sync(0xffffffffu, r0, 8); r0 += __shfl_xor_sync(0xffffffffu, r0, 16);
-            r1 += __shfl_xor_sync(0xffffffffu, r1, 8); r1 += __shfl_xor_sync(0xffffffffu, r1, 16);
+            if constexpr (!MMA1) {
+                r0 = acc[0] + acc[1], r1 = acc[2] + acc[3];
+                r0 += __shfl_xor_sync(0xffffffffu, r0, 8); r0 += __shfl_xor_sync(0xffffffffu, r0, 16);
+                r1 += __shfl_xor_sync(0xffffffffu, r1, 8); r1 += __shfl_xor_sync(0xffffffffu, r1, 16);
+            }
             if (tig == 0) {
                 if (whole) {
                     Y[rb * 16 + gid] = __float2half_rn(r0);
@@ -519,7 +595,7 @@ inline int ring_error_fetch() {
 template <int BITS, int MODE, int MT>
 pot_status_t launch_ring(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                          const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
-    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1);
+    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, MODE == RG_POT_FMA || MODE == RG_UINT_FMA);
     auto run = [&](auto kernel) -> pot_status_t {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
             return POT_ERR_CUDA;
@@ -529,7 +605,7 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
                           (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
                           (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
     };
-    if constexpr (MODE != RG_POT_MMA) {
+    if constexpr (MODE == RG_POT_FMA || MODE == RG_UINT_FMA) {
         if (p.x_in_smem && p.x_wide) return run(ring_kernel<BITS, MODE, MT, 2>);
     }
     if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, 1>);
