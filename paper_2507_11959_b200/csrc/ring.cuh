@@ -27,15 +27,18 @@
 
 namespace pot {
 
-constexpr int RG_CONSUMERS = 15;
-constexpr int RG_THREADS = (RG_CONSUMERS + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3 };
+
+enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3, RG_POT_MMA1W = 4 };
 
 constexpr int RG_Q = 5;  // steps per ring slot (one bulk copy) = warps per consumer group
-constexpr int RG_GROUPS = RG_CONSUMERS / RG_Q;  // slot m is consumed by group m % RG_GROUPS, warp i of it takes step i
-static_assert(RG_GROUPS * RG_Q == RG_CONSUMERS, "consumer warps must split into whole groups");
+// Consumer groups per CTA: slot m is consumed by group m % groups, warp i of it takes step i.  The tensor-core
+// GEMV needs fewer registers per thread, so one more group of warps fits (RG_POT_MMA1W); whether that pays
+// depends on how evenly the CTA's steps divide among the warps, see launch_gemv_mma.
+__host__ __device__ constexpr int rg_groups(int mode) { return mode == RG_POT_MMA1W ? 4 : 3; }
+__host__ __device__ constexpr int rg_consumers(int mode) { return rg_groups(mode) * RG_Q; }
+__host__ __device__ constexpr int rg_threads(int mode) { return (rg_consumers(mode) + 1) * 32; }
 __host__ __device__ constexpr int rg_unit_bytes(int bits) { return 256 * bits; }
 __host__ __device__ constexpr int rg_slot_bytes(int bits) { return RG_Q * 4 * rg_unit_bytes(bits); }
 
@@ -53,7 +56,7 @@ struct RingPlan {
     size_t ws_bytes;
 };
 
-inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bool wide_ok = true) {
+inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bool wide_ok = true, int groups = 3) {
     RingPlan p;
     const int64_t nrb = N / 16, ncb = K / 128;
     p.spr = (int)((ncb + 3) / 4);
@@ -75,7 +78,7 @@ inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bo
     // A slot that is reused must always come back to the same group of consumer warps (see the kernel):
     // the ring length is a multiple of the number of groups unless it holds the CTA's whole share.
     if (st >= slots_needed) st = slots_needed;
-    else st = st / RG_GROUPS * RG_GROUPS;
+    else st = st / groups * groups;
     if (st < 1) st = 1;
     p.stages = (int)st;
     p.smem_bytes = 1024 + p.x_bytes + p.cmb_bytes + (size_t)p.stages * (size_t)rg_slot_bytes(bits);
@@ -143,7 +146,8 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(RG_CONSUMERS * 32) : "memory"); }
+template <int NC>
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NC * 32) : "memory"); }
 
 __device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
     asm("{\n\t"
@@ -183,7 +187,7 @@ __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
 // of the A fragment -- and the MMA adds up the four quarters, so there is no cross-lane reduction and the
 // multiply-accumulate costs one instruction per 256 weights instead of one per weight.
 template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = staged packed, 2 = staged wide
-__global__ void __launch_bounds__(RG_THREADS, 1)
+__global__ void __launch_bounds__(rg_threads(MODE), 1)
 ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
             int64_t N, int64_t K, int G, int spr, int64_t total_steps, int stages, int x_bytes, int cmb_bytes,
             const __half* __restrict__ X, int M, __half* __restrict__ Y, float* __restrict__ partial,
@@ -193,7 +197,8 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     constexpr bool XWIDE = (XMODE == 2);
     constexpr bool MMA = (MODE == RG_POT_MMA);
     constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
-    constexpr bool MMA1 = (MODE == RG_POT_MMA1);
+    constexpr int RG_CONSUMERS = rg_consumers(MODE), RG_GROUPS = rg_groups(MODE);
+    constexpr bool MMA1 = (MODE == RG_POT_MMA1 || MODE == RG_POT_MMA1W);
     constexpr int TOK = MMA ? 8 * MT : 1;
     constexpr int SLOT = rg_slot_bytes(BITS);
     constexpr int UB = rg_unit_bytes(BITS);
@@ -324,7 +329,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                 dst[i] = v;
             }
         }
-        consumer_bar_sync();
+        consumer_bar_sync<RG_CONSUMERS>();
     }
 
     // per-lane activation row pointers for the tensor path (token = 8*mt + gid), hoisted out of the loop
@@ -595,13 +600,14 @@ inline int ring_error_fetch() {
 template <int BITS, int MODE, int MT>
 pot_status_t launch_ring(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                          const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
-    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, MODE == RG_POT_FMA || MODE == RG_UINT_FMA);
+    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, MODE == RG_POT_FMA || MODE == RG_UINT_FMA,
+                                 rg_groups(MODE));
     auto run = [&](auto kernel) -> pot_status_t {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
             return POT_ERR_CUDA;
         unsigned* counters = (unsigned*)workspace;
         float* partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
-        return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(RG_THREADS), p.smem_bytes, s, (const uint4*)packed,
+        return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(rg_threads(MODE)), p.smem_bytes, s, (const uint4*)packed,
                           (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
                           (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
     };
@@ -610,6 +616,18 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
     }
     if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, 1>);
     return run(ring_kernel<BITS, MODE, MT, 0>);
+}
+
+// GEMV on the warp-level tensor-core path with 15 or 20 consumer warps: a warp works through whole steps, so the
+// time is (steps per warp, rounded up) x (time per step, about 1.2 x longer when 20 warps share the SM).
+template <int BITS>
+pot_status_t launch_gemv_mma(const void* packed, const void* scales, int64_t N, int64_t K, int group, const void* x, void* y,
+                             void* workspace, int* err, cudaStream_t s) {
+    const RingPlan p = plan_ring(N, K, 1, BITS, 1, false, 3);
+    const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
+    const double t3 = (double)((per_cta + 14) / 15), t4 = 1.2 * (double)((per_cta + 19) / 20);
+    if (t4 < t3) return launch_ring<BITS, RG_POT_MMA1W, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, err, s);
+    return launch_ring<BITS, RG_POT_MMA1, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, err, s);
 }
 
 }  // namespace pot
