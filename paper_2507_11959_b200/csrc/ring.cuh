@@ -220,11 +220,9 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         return (int64_t)rbq * ncb + 4 * (int64_t)((uint32_t)g - rbq * (uint32_t)spr);
     };
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(smem_u32(&bars[s]), 1);                // full: the producer's expect_tx arrival
-            mbar_init(smem_u32(&bars[stages + s]), RG_Q);    // empty: one arrival per consumed step
-        }
+    if (threadIdx.x < stages) {  // one thread per ring slot
+        mbar_init(smem_u32(&bars[threadIdx.x]), 1);                // full: the producer's expect_tx arrival
+        mbar_init(smem_u32(&bars[stages + threadIdx.x]), RG_Q);    // empty: one arrival per consumed step
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     unsigned* cmb_cnt = reinterpret_cast<unsigned*>(cmb + (size_t)(nsteps + 1) * 16 * TOK);
