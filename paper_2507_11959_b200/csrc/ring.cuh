@@ -63,8 +63,9 @@ inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bo
     p.total_steps = nrb * p.spr;
     p.grid = (int)(p.total_steps < kSmCount ? p.total_steps : kSmCount);
     p.x_wide = wide_ok && (tok == 1) && (size_t)K * 4 <= 48 * 1024;
-    const size_t xb = (size_t)M * (size_t)K * (p.x_wide ? 4 : 2);
-    p.x_in_smem = xb <= 64 * 1024;
+    // the small-batch mode stages a full tile of eight tokens (fragment order), whatever M is
+    const size_t xb = (size_t)(tok > 1 ? tok : M) * (size_t)K * (p.x_wide ? 4 : 2);
+    p.x_in_smem = xb <= (tok > 1 ? 96 : 64) * 1024;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
     const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
     // per step one slot of 16*tok floats, plus one counter per local row block
@@ -199,6 +200,8 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
     constexpr int RG_CONSUMERS = rg_consumers(MODE), RG_GROUPS = rg_groups(MODE);
     constexpr bool MMA1 = (MODE == RG_POT_MMA1 || MODE == RG_POT_MMA1W);
+    constexpr bool TC = MMA || MMA1;  // tensor-core modes: lane (gid, tig) owns quarter tig of rows gid and gid + 8
+    static_assert(!MMA || MT == 1, "one tile of eight tokens");
     constexpr int TOK = MMA ? 8 * MT : 1;
     constexpr int SLOT = rg_slot_bytes(BITS);
     constexpr int UB = rg_unit_bytes(BITS);
@@ -255,15 +258,15 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     }
 
     // -------------------- consumers --------------------------------------------------------------------
-    const int gid = (MMA || MMA1) ? (lane >> 2) : (lane & 7);
-    const int tig = (MMA || MMA1) ? (lane & 3) : (lane >> 3);
+    const int gid = TC ? (lane >> 2) : (lane & 7);
+    const int tig = TC ? (lane & 3) : (lane >> 3);
     const int gpr = (int)(K / G);
     const int spg = 128 / G;
 
     // scales (and zero-points) of a step are fetched one step ahead, straight from global memory.  The
     // buffers keep the raw 16-bit loads: any arithmetic on them here would make the warp wait for the load.
-    // RG_POT_MMA1: the scale of this lane's quarter, for both rows and the four units of a step
-    uint32_t sc1[2][MMA1 ? 8 : 1];
+    // tensor-core modes: the scale of this lane's quarter, for both rows and the four units of a step
+    uint32_t sc1[2][TC ? 8 : 1];
     auto load_scales_mma1 = [&](int64_t rb, int c, int buf) {
         // one 64-bit address per step; the eight loads use constant offsets from it
         const uint16_t* s0 = scales + (rb * 16 + gid) * gpr + (int64_t)c * (4 * spg) + (spg == 2 ? (tig >> 1) : 0);
@@ -280,7 +283,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     };
     uint32_t sc[2][2][2], zp[2][2][2];
     auto load_scales = [&](int64_t rb, int c, int buf) {
-        if constexpr (MMA1) { load_scales_mma1(rb, c, buf); return; }
+        if constexpr (TC) { load_scales_mma1(rb, c, buf); return; }
         const int64_t cb = 4 * (int64_t)c + tig;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -313,32 +316,43 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     if constexpr (XSMEM) {
         uint4* dst = reinterpret_cast<uint4*>(smem + 1024);
         const uint4* src = reinterpret_cast<const uint4*>(X);
-        const int n16 = (int)((int64_t)M * K / 8);
-        for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) {
-            const uint4 v = __ldg(src + i);
-            if constexpr (XWIDE) {
-                dst[2 * i] = make_uint4(v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16);
-                dst[2 * i + 1] = make_uint4(v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16);
-            } else if constexpr (MMA1) {
-                // chunk (quarter t, part j) of a unit goes to position j * 4 + t: the four lanes tig = 0..3 then
-                // read 64 contiguous bytes
-                dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v;
-            } else {
-                dst[i] = v;
+        if constexpr (MMA) {
+            // 16-byte chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * 8 + token: the 32
+            // lanes of a warp (token = gid, t = tig) then read 512 contiguous bytes.  Tokens >= M stay unwritten:
+            // their columns of the product are never delivered.
+            const int kc = (int)(K / 8);
+            constexpr int NT = RG_CONSUMERS * 32;
+            for (int token = 0; token < M; ++token)
+                for (int c0 = threadIdx.x; c0 < kc; c0 += 4 * NT) {  // four loads in flight per thread
+                    uint4 v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (c0 + i * NT < kc) v[i] = __ldg(src + (int64_t)token * kc + c0 + i * NT);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int cc = c0 + i * NT;
+                        if (cc < kc) dst[((((cc >> 4) * 4 + (cc & 3)) * 4 + ((cc >> 2) & 3)) << 3) + token] = v[i];
+                    }
+                }
+        } else {
+            const int n16 = (int)(K / 8);
+            for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) {
+                const uint4 v = __ldg(src + i);
+                if constexpr (XWIDE) {
+                    dst[2 * i] = make_uint4(v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16);
+                    dst[2 * i + 1] = make_uint4(v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16);
+                } else if constexpr (MMA1) {
+                    // chunk (quarter t, part j) of a unit goes to position j * 4 + t: the four lanes tig = 0..3 then
+                    // read 64 contiguous bytes
+                    dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v;
+                } else {
+                    dst[i] = v;
+                }
             }
         }
         consumer_bar_sync<RG_CONSUMERS>();
     }
 
-    // per-lane activation row pointers for the tensor path (token = 8*mt + gid), hoisted out of the loop
-    const uint4* xrow[MT];
-    bool xrow_ok[MT];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        const int token = 8 * mt + gid;
-        xrow_ok[mt] = MMA && token < M;
-        xrow[mt] = (XSMEM ? xs : reinterpret_cast<const uint4*>(X)) + (xrow_ok[mt] ? (int64_t)token * (K / 8) : 0);
-    }
     const int64_t rb_first = g_begin / spr;
     int m = grp, slot = grp % stages;        // this warp's current slot fill, ring slot and barrier phase
     uint32_t phase = (uint32_t)((grp / stages) & 1);
@@ -357,7 +371,8 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             if (err && lane == 0) atomicCAS(err, 0, 2 | (m << 8) | (warp << 16) | (j << 24));
         }
         float r0 = 0.f, r1 = 0.f;  // RG_POT_MMA1: the sums of rows gid and gid + 8
-        if constexpr (MMA1) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (TC) {
             // units between the slot's first step (wig steps back) and this one, without divisions
             int64_t rb_s = rb;
             int c_s = c - wig;
@@ -370,6 +385,24 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             for (int i = 0; i < 2; ++i)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+            // RELEASE_EARLY: the step's records are copied to registers and the slot is handed back before the
+            // arithmetic (the small-batch mode has few slots, its activations take most of the shared memory)
+            constexpr bool RELEASE_EARLY = MMA;
+            uint32_t wreg[RELEASE_EARLY ? 4 : 1][2][BITS];
+            if constexpr (RELEASE_EARLY) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int k = 0; k < BITS; ++k) {
+                            wreg[u][h][k] = 0u;
+                            if (4 * (int64_t)c + u < ncb)
+                                wreg[u][h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
+                        }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
+            }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int64_t cbu = 4 * (int64_t)c + u;
@@ -378,14 +411,26 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
-                        for (int k = 0; k < BITS; ++k)
-                            w[h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
-                    uint32_t xq[16];  // the 32 activations of quarter tig: the B fragments of eight MMAs
-                    {
+                        for (int k = 0; k < BITS; ++k) {
+                            if constexpr (RELEASE_EARLY) w[h][k] = wreg[u][h][k];
+                            else w[h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
+                        }
+                    uint32_t xq[16];  // 32 activations of quarter tig (of token gid): the B fragments of eight MMAs
+                    if constexpr (MMA1) {
                         const uint4* xp = (XSMEM ? xs : reinterpret_cast<const uint4*>(X)) + cbu * 16 + (XSMEM ? tig : tig * 4);
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const uint4 v = XSMEM ? xp[4 * i] : __ldg(xp + i);
+                            xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
+                        }
+                    } else {
+                        const uint4* xp = XSMEM ? xs + (cbu * 16 + tig) * 8 + gid
+                                                : reinterpret_cast<const uint4*>(X) + (gid < M ? (int64_t)gid * (K / 8) : 0) + cbu * 16 + tig * 4;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (XSMEM) v = xp[32 * i];
+                            else if (gid < M) v = __ldg(xp + i);
                             xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
                         }
                     }
@@ -397,13 +442,16 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                         rg_mma(acc1[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
-            r0 = acc1[0][0] + acc1[1][0];   // every column of the product holds the same sums
+            if constexpr (!RELEASE_EARLY) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
+            }
+            r0 = acc1[0][0] + acc1[1][0];   // GEMV: every column of the product holds the same sums
             r1 = acc1[0][2] + acc1[1][2];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e] = acc1[0][e] + acc1[1][e];
         }
-        float acc[MMA ? 4 * MT : 4];
-        if constexpr (!MMA1) {
+        if constexpr (!TC) {
         uint32_t rec[2][NW];
         {
             // records are fetched with lane (column block, row) = (lane / 8, lane % 8): 8 lanes read 128
@@ -424,21 +472,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                     if (fvalid) q = unit[t * 16 + fgid + 8 * h];
                     rec[h][4 * t + 0] = q.x; rec[h][4 * t + 1] = q.y; rec[h][4 * t + 2] = q.z; rec[h][4 * t + 3] = q.w;
                 }
-            if constexpr (MMA) {
-                // hand the records over to the lanes that own them in the MMA fragment layout
-                const int src = ((lane & 3) << 3) | (lane >> 2);
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int i = 0; i < NW; ++i) rec[h][i] = __shfl_sync(0xffffffffu, rec[h][i], src);
-            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
 
-#pragma unroll
-        for (int i = 0; i < (MMA ? 4 * MT : 4); ++i) acc[i] = 0.f;
-        if (!MMA) {
+        {
             if (valid) {
 #pragma unroll
                 for (int T = 0; T < 4; ++T) {
@@ -467,29 +505,6 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                             else rg_fma2(acc[2 * h], acc[2 * h + 1], w2[p], xw[p]);
                         }
                     }
-                }
-            }
-        } else {
-#pragma unroll
-            for (int T = 0; T < 4; ++T) {
-                uint32_t w0[16], w1[16];
-                potl::pot_decode32<BITS>(rec[0], T, sc[buf][0][T >> 1] * 0x10001u, w0);
-                potl::pot_decode32<BITS>(rec[1], T, sc[buf][1][T >> 1] * 0x10001u, w1);
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    uint32_t xw[16];
-                    const bool xok = valid && xrow_ok[mt];
-                    const uint4* xp = xrow[mt] + cb * 16 + 4 * T;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 v = make_uint4(0, 0, 0, 0);
-                        if (xok) v = XSMEM ? xp[i] : __ldg(xp + i);
-                        xw[4 * i + 0] = v.x; xw[4 * i + 1] = v.y; xw[4 * i + 2] = v.z; xw[4 * i + 3] = v.w;
-                    }
-                    float(&a)[4] = *reinterpret_cast<float(*)[4]>(&acc[4 * mt]);
-#pragma unroll
-                    for (int st = 0; st < 8; ++st)
-                        rg_mma(a, w0[2 * st], w1[2 * st], w0[2 * st + 1], w1[2 * st + 1], xw[2 * st], xw[2 * st + 1]);
                 }
             }
         }
@@ -529,7 +544,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                     if (whole) {
                         if (token < M) Y[(int64_t)token * N + rb * 16 + row] = __float2half_rn(acc[4 * mt + e]);
                     } else {
-                        pslot[token * 16 + row] = acc[4 * mt + e];
+                        if (token < M) pslot[token * 16 + row] = acc[4 * mt + e];
                     }
                 }
         }
@@ -548,7 +563,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             if (prev == (unsigned)spr - 1u) {  // this warp delivered the last slot of the row block
                 if (local) __threadfence_block(); else __threadfence();
                 const float* first = local ? cmb + (size_t)(rb_g0 - g_begin) * (16 * TOK) : partial + rb_g0 * (16 * TOK);
-                for (int e = lane; e < 16 * TOK; e += 32) {
+                for (int e = lane; e < 16 * (MMA ? M : 1); e += 32) {
                     const int row = e & 15, token = e >> 4;
                     float sum = 0.f;
                     if (local) {
