@@ -275,7 +275,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": value / world / peaks["hbm_gbs"], "frac_of_8TBs_nominal": value / world / 8000.0,
-                     "peak_source": peaks["source"], "kernel": "ring_kernel<3, RG_POT_FMA, 1> (decode GEMV, tiled layout)",
+                     "peak_source": peaks["source"], "kernel": "ring_kernel<3, RG_POT_MMA1|RG_POT_MMA1W, 1> (decode GEMV on mma.sync, tiled layout)",
                      "per_launch_us": ms * 1e3 / max(1, launches_per_step),
                      "algorithmic_bytes_per_launch": bytes3 / max(1, launches_per_step),
                      # dram__bytes_read+write per launch from the ncu capture of the 12288x4096 launch

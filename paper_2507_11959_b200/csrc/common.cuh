@@ -37,6 +37,15 @@ constexpr int kSmCount = 148;  // B200: 2 dies x 74 SMs
 // Launch with programmatic stream serialization: the kernel may start while the previous kernel
 // in the stream is still draining; it must execute griddepcontrol.wait before touching anything
 // the previous kernel wrote (and before writing anything the previous kernel may still read).
+// Largest dynamic shared memory a CTA may ask for on sm_100a.  Kernels opt in to this maximum rather than to the
+// size of the current launch: a launch recorded in a CUDA graph must still fit the function's attribute when the
+// graph is replayed, whatever other shapes were launched in between.
+constexpr int kMaxDynamicSmem = 227 * 1024;
+template <typename K>
+inline bool allow_max_dynamic_smem(K kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess;
+}
+
 template <typename... Args>
 inline pot_status_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};

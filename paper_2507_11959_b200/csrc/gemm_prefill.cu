@@ -318,7 +318,7 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
     const bool deep = (int64_t)grid.x * grid.y <= 2 * kSmCount;  // too few tiles to fill two CTAs per SM anyway
     auto run = [&](auto kernel, int stages) -> pot_status_t {
         const size_t smem = pf_smem_bytes(stages);
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return POT_ERR_CUDA;
+        if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (__half*)Y, prefill_error_ptr());
     };

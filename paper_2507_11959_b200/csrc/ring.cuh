@@ -616,8 +616,7 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
     const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, MODE == RG_POT_FMA || MODE == RG_UINT_FMA,
                                  rg_groups(MODE));
     auto run = [&](auto kernel) -> pot_status_t {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
-            return POT_ERR_CUDA;
+        if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         unsigned* counters = (unsigned*)workspace;
         float* partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
         return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(rg_threads(MODE)), p.smem_bytes, s, (const uint4*)packed,
