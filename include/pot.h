@@ -122,10 +122,13 @@ pot_status_t pot_validate_scales(const void* scales_f16, int64_t count, int bits
  *
  * Tiled layout: the matrix is cut into units of 16 rows x 128 columns (one unit per row block
  * rb = i/16 and column block cb = k/128, stored in [rb][cb] order, 16*128*n/8 bytes each).
- * A unit holds n "planes" of 256 bytes; plane t stores, for row r of the unit, the 16-byte
- * word t of that row's 128-code record at byte offset t*256 + r*16.  The record of one row
- * (n 16-byte words = 4n 32-bit words) arranges its 128 codes so that codes 2p and 2p+1 of an
- * 8-code block sit 16 bits apart in one 32-bit word (see csrc/layout.cuh for the bit map).
+ * A unit holds n "planes" of 256 bytes; plane k stores, for row r of the unit, 16 bytes at
+ * offset k*256 + r*16: word k of each of the four 32-column quarters of that row's 128-code
+ * record (record word index 4k + quarter).  Inside a word the PoT codes are laid out as byte
+ * lanes shaped like an 8-bit float (exponent bits from bit 2, sign at bit 7, after a rotation),
+ * so that one rotate + one mask extract four codes and one multiply-add per pair places them
+ * in the FP16 exponent / sign fields; the uniform codes are plain n-bit fields with the two
+ * codes of a pair 16 bits apart.  csrc/layout.cuh has the bit map; pot_layout_bit reports it.
  */
 pot_status_t pot_repack(const void* src, void* dst, int64_t N, int64_t K, int bits, int direction,
                         void* stream);
@@ -146,10 +149,12 @@ pot_status_t pot_dequant(const void* packed, const void* scales_f16, int64_t N, 
 
 /*
  * pot_gemv -- batch-1 decode: y = W~ x with W~ the FP16 reconstruction (Eq. 1), FP32
- * accumulation, FP16 output.  CUDA-core kernel: codes are decoded in registers with the
- * integer-add trick, lanes reduce over K with warp shuffles, and K is split across CTAs when N
- * alone cannot fill the GPU (partials in `workspace`, summed in a fixed order, so results are
- * bit-identical run to run).
+ * accumulation, FP16 output.  Codes are decoded in registers with the integer-add trick (Sec.
+ * 4.2).  Tiled layout: a persistent kernel streams the codes through a shared-memory ring, the
+ * decoded FP16 weights are the A fragments of warp-level tensor-core MMAs whose B columns all
+ * hold x, and the matrix is split evenly across the SMs (partial sums of a row block that spans
+ * CTAs go through `workspace` and are added in a fixed order, so results are bit-identical run
+ * to run).  Canonical layout: a CUDA-core kernel with warp-shuffle reduction.
  *   x_f16 [K], y_f16 [N]; workspace >= pot_gemv_workspace_bytes(N,K,bits,group), 16-byte aligned
  *   (may be NULL when that size is 0).  `layout` says how `packed` is arranged.
  */

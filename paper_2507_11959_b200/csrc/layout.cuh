@@ -11,7 +11,7 @@
 // of an 8-bit float with five exponent bits: exponent bits from bit 2 upwards, sign at bit 7
 // (five above the exponent's low bit), after a rotation of the word:
 //   * as FP8 operand : (rot(w) & mask) | 0x40..  is the byte pattern of +-2^(E+1) -- one
-//                      logic operation per four weights, consumed by the FP8 tensor-core MMA;
+//                      logic operation per four weights (no kernel in this tree consumes that form yet);
 //   * as FP16 pair   : (rot(w) & mask16) * 2^8 + scale  (lanes 0, 2)  and
 //                      (rot(w) & mask16 << 8) + scale   (lanes 1, 3)  -- the mask / shift /
 //                      integer add into the scale's bit pattern of Sec. 4.2 of the paper.
@@ -150,21 +150,6 @@ struct PotLanes<4> {
         }
     }
 };
-
-// Quarter -> eight words of four FP8 (five exponent bits, two mantissa bits) bytes: byte lane l of
-// word i is +-2^(E+1) for column 4i + perm[l] of the quarter.  The constant 0x40 per byte sets
-// the exponent field to 16 + E.
-template <int BITS>
-__device__ __forceinline__ void pot_decode32_f8(const uint32_t (&w)[BITS], uint32_t (&dw)[8]) {
-    using L = PotLanes<BITS>;
-    uint32_t d[8];
-    L::rotate(w, d);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        if (L::LOW7 && i == 7) dw[i] = mad(d[i] & (L::MASK >> 2), 4u, 0x40404040u);
-        else dw[i] = (d[i] & L::MASK) | 0x40404040u;
-    }
-}
 
 // Decode 32 consecutive codes (16 pairs): quarter T (0..3) of a record held in registers
 // (rec[STRIDE * k + T] = word k of the quarter; STRIDE = 4 for a whole record).  out[p] = bit pattern of half2{ w~[2p], w~[2p+1] }:
