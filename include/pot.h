@@ -201,7 +201,11 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
  * accumulation, FP16 output.  M <= 8 (decode batches) runs a bandwidth-bound tensor-core
  * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the
  * tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
- * accumulators in tensor memory.  The prefill kernel requires layout == POT_LAYOUT_TILED.
+ * accumulators in tensor memory; when the output tiles cover less than half of the SMs it
+ * splits K across CTAs (FP32 partial sums and arrival counters in `workspace`, added in a fixed
+ * order).  The tcgen05 kernel requires layout == POT_LAYOUT_TILED.
+ *   workspace >= pot_gemm_workspace_bytes(M,N,K,bits,group), 16-byte aligned, zero before its
+ *   first use (the kernels leave the counters at zero); may be NULL when that size is 0.
  */
 pot_status_t pot_gemm(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
                       int group, pot_layout_t layout, const void* X_f16, int64_t M, void* Y_f16,

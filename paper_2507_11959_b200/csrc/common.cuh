@@ -43,7 +43,10 @@ constexpr int kSmCount = 148;  // B200: 2 dies x 74 SMs
 constexpr int kMaxDynamicSmem = 227 * 1024;
 template <typename K>
 inline bool allow_max_dynamic_smem(K kernel) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess;
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return false;
+    const int room = kMaxDynamicSmem - (int)fa.sharedSizeBytes;  // static shared memory counts against the same limit
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, room) == cudaSuccess;
 }
 
 template <typename... Args>

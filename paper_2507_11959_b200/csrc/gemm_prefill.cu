@@ -83,7 +83,8 @@ template <int BITS, int PF_STAGES>
 __global__ void __launch_bounds__(PF_THREADS, PF_STAGES == 2 ? 2 : 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
-                        __half* __restrict__ Y, int* __restrict__ err) {
+                        __half* __restrict__ Y, float* __restrict__ partial, unsigned* __restrict__ counters,
+                        int* __restrict__ err) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -97,8 +98,11 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.x * (PF_BM * PF_MT), n0 = (int64_t)blockIdx.y * PF_BN;
-    const int nkb = (int)(K / PF_BK);
     const int64_t ncb = K / 128;
+    // split-K (few tiles, small M): CTA z of gridDim.z owns column blocks [cb0, cb1), two stages each
+    const int64_t cb0 = (int64_t)blockIdx.z * ncb / gridDim.z, cb1 = ((int64_t)blockIdx.z + 1) * ncb / gridDim.z;
+    const int nkb = (int)(2 * (cb1 - cb0));
+    const int kb0 = (int)(2 * cb0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
@@ -131,7 +135,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
 #pragma unroll
                 for (int mt = 0; mt < PF_MT; ++mt)
-                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, kb * PF_BK, (int)m0 + mt * PF_BM, full(s));
+                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
             }
         }
     } else if (warp == 1) {
@@ -180,13 +184,13 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         uint32_t sc2[PF_DEPTH];
         auto load = [&](int kb, int buf) {
             if (row_ok) {
-                const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + (kb >> 1)) * (16 * BITS));
+                const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cb0 + (kb >> 1)) * (16 * BITS));
 #pragma unroll
                 for (int t = 0; t < BITS; ++t) {
                     const uint2 q = __ldg(unit + (t * 16 + r) * 2 + grp);
                     rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
                 }
-                const int64_t so = n * gpr + (int64_t)(kb >> 1) * spg + (spg == 2 ? grp : 0);
+                const int64_t so = n * gpr + (cb0 + (kb >> 1)) * spg + (spg == 2 ? grp : 0);
                 sc2[buf] = (uint32_t)__ldg(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
@@ -239,6 +243,25 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
         const int mt = (warp - 2) >> 2;           // warps 2..5 read accumulator 0, warps 6..9 accumulator 1
         const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
+        const int splits = (int)gridDim.z;
+        auto store_row = [&](const uint32_t (&v)[32], int col) {  // 32 FP32 sums of one token -> FP16 -> Y
+            __half* dst = Y + token * N + n0 + col;
+            if (n0 + col + 32 <= N) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __half2 h = __floats2half2_rn(__uint_as_float(v[8 * i + 2 * j]), __uint_as_float(v[8 * i + 2 * j + 1]));
+                        o[j] = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(dst + 8 * i) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            } else {
+                for (int i = 0; i < 32; ++i)
+                    if (n0 + col + i < N) dst[i] = __float2half_rn(__uint_as_float(v[i]));
+            }
+        };
 #pragma unroll
         for (int cc = 0; cc < PF_BN / 32; ++cc) {
             const int col = cc * 32;
@@ -246,22 +269,52 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(mt * PF_BN + col), v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             if (token < M) {
-                __half* dst = Y + token * N + n0 + col;
-                if (n0 + col + 32 <= N) {
+                if (splits == 1) {
+                    store_row(v, col);
+                } else {  // this split's partial sums, [split][token][feature] FP32 (N % 16 == 0: whole 16-byte pieces)
+                    float* dst = partial + ((int64_t)blockIdx.z * M + token) * N + n0 + col;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t o[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const __half2 h = __floats2half2_rn(__uint_as_float(v[8 * i + 2 * j]), __uint_as_float(v[8 * i + 2 * j + 1]));
-                            o[j] = *reinterpret_cast<const uint32_t*>(&h);
-                        }
-                        *reinterpret_cast<uint4*>(dst + 8 * i) = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                } else {
-                    for (int i = 0; i < 32; ++i)
-                        if (n0 + col + i < N) dst[i] = __float2half_rn(__uint_as_float(v[i]));
+                    for (int i = 0; i < 8; ++i)
+                        if (n0 + col + 4 * i < N)
+                            *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
+            }
+        }
+        if (splits > 1) {
+            // The CTA that delivers the last split of a tile (an arrival counter tells it) adds the splits in
+            // ascending order -- the result does not depend on timing -- and writes Y.
+            __shared__ unsigned s_prev;
+            __threadfence();
+            asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
+            const unsigned tile = blockIdx.y * gridDim.x + blockIdx.x;
+            if (threadIdx.x == 64) s_prev = atomicAdd(&counters[tile], 1u);
+            asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
+            if (s_prev == (unsigned)splits - 1u) {
+                __threadfence();
+                if (token < M) {
+#pragma unroll 1
+                    for (int cc = 0; cc < PF_BN / 32; ++cc) {
+                        const int col = cc * 32;
+                        if (n0 + col >= N) break;
+                        float sum[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) sum[i] = 0.f;
+                        for (int z = 0; z < splits; ++z) {
+                            const float* src = partial + ((int64_t)z * M + token) * N + n0 + col;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (n0 + col + 4 * i < N) {
+                                    const float4 t = __ldcg(reinterpret_cast<const float4*>(src + 4 * i));
+                                    sum[4 * i] += t.x; sum[4 * i + 1] += t.y; sum[4 * i + 2] += t.z; sum[4 * i + 3] += t.w;
+                                }
+                        }
+                        uint32_t v[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(sum[i]);
+                        store_row(v, col);
+                    }
+                }
+                if (threadIdx.x == 64) counters[tile] = 0u;  // leave the workspace ready for the next call
             }
         }
     }
@@ -296,13 +349,36 @@ bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group
     // TMA needs the X row pitch (2K bytes) to be a multiple of 16 -- implied by K % 128 == 0 -- and 32-bit box coordinates
     return M > 0 && N % 16 == 0 && K % 128 == 0 && M < (int64_t(1) << 31) && K < (int64_t(1) << 31);
 }
-size_t gemm_prefill_workspace(int64_t, int64_t, int64_t, int, int) { return 0; }
+// Split-K when the tiles cover less than half of the SMs (small M, narrow N): enough CTAs for two per SM, at least
+// four column blocks each.  (With more tiles than that the per-stage hand-off latency, which two co-resident
+// CTAs share, bounds the kernel either way and splitting only adds the reduction.)
+static int prefill_splits(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)) * ((N + PF_BN - 1) / PF_BN);
+    if (2 * tiles > kSmCount) return 1;
+    int64_t s = 2 * kSmCount / tiles;
+    const int64_t max_by_k = (K / 128) / 4;
+    if (s > max_by_k) s = max_by_k;
+    if (s > 16) s = 16;
+    return s < 1 ? 1 : (int)s;
+}
+static size_t prefill_counter_bytes(int64_t M, int64_t N) {
+    const int64_t tiles = ((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)) * ((N + PF_BN - 1) / PF_BN);
+    return ((size_t)tiles * 4 + 255) / 256 * 256;
+}
+// arrival counters (must start at zero; the kernel leaves them at zero) + [splits][M][N] FP32 partial sums
+size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) {
+    const int s = prefill_splits(M, N, K);
+    return s == 1 ? 0 : prefill_counter_bytes(M, N) + (size_t)s * (size_t)M * (size_t)N * 4;
+}
 
 static int* prefill_error_ptr();
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s) {
-    (void)workspace; (void)ws_bytes;
+    const int splits = prefill_splits(M, N, K);
+    if (splits > 1 && (!workspace || ws_bytes < gemm_prefill_workspace(M, N, K, bits, group))) return POT_ERR_WORKSPACE;
+    unsigned* counters = (unsigned*)workspace;
+    float* partial = splits > 1 ? (float*)((char*)workspace + prefill_counter_bytes(M, N)) : nullptr;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return POT_ERR_CUDA;
     CUtensorMap xmap;
@@ -314,13 +390,15 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
-    const dim3 grid((unsigned)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)), (unsigned)((N + PF_BN - 1) / PF_BN)), block(PF_THREADS);
-    const bool deep = (int64_t)grid.x * grid.y <= 2 * kSmCount;  // too few tiles to fill two CTAs per SM anyway
+    const dim3 grid((unsigned)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)), (unsigned)((N + PF_BN - 1) / PF_BN), (unsigned)splits),
+        block(PF_THREADS);
+    // too few CTAs to fill two per SM: one CTA per SM with the deeper pipeline
+    const bool deep = (int64_t)grid.x * grid.y * grid.z <= 2 * kSmCount && splits == 1;
     auto run = [&](auto kernel, int stages) -> pot_status_t {
         const size_t smem = pf_smem_bytes(stages);
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
-                          (__half*)Y, prefill_error_ptr());
+                          (__half*)Y, partial, counters, prefill_error_ptr());
     };
     if (deep) {
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4>, 4);

@@ -16,7 +16,7 @@ def B():
 
 
 # (M, N, K): one exact tile; ragged M and N with several K blocks; several tiles in both directions
-SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152)]
+SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20, 256, 4096)]  # the last two run split-K
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -30,6 +30,25 @@ def test_prefill_gemm_matches_oracle(B, oracle, bits, G):
         assert B.pot_debug_errors() == (0, 0, 0)
         ok, worst, tight = gate(bits_of(Yg), Y, A)
         assert ok and tight < 4.0, (M, N, K, worst, tight)
+
+
+def test_split_k_workspace_is_reusable(B, oracle):
+    """Few tiles and a deep K: the kernel splits K (8 ways here), adds the splits in a fixed order and leaves its
+    arrival counters at zero -- two calls on one workspace give the same bits, equal to the oracle within the gate."""
+    bits, G, M, N, K = 3, 128, 40, 384, 4096
+    c = PotCase(N, K, bits, G, dist="t5", seed=(5, 77))
+    X = synth.activations(synth.rng_for(5, 177), M, K, outliers=True)
+    Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
+    need = B.pot_gemm_workspace_bytes(M, N, K, bits, G)
+    assert need > 0
+    ws = B.new_workspace(need)
+    dX = f16_dev(X)
+    y1 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
+    y2 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
+    assert B.pot_debug_errors() == (0, 0, 0)
+    assert np.array_equal(y1, y2)
+    ok, worst, tight = gate(y1, Y, A)
+    assert ok and tight < 4.0, (worst, tight)
 
 
 @pytest.mark.parametrize("bits", [3])
