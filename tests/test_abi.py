@@ -46,7 +46,9 @@ def test_size_helpers(L):
     ws = L.pot_gemv_workspace_bytes(4096, 11008, 3, 128)
     assert ws == 1024 + 256 * 22 * 16 * 4 and ws % 16 == 0
     assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
-    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 0   # M > 8 runs the tcgen05 kernel: no scratch
+    # M > 8 runs the tcgen05 kernel: no scratch unless few tiles make it split K (32 tiles -> 9 splits here)
+    assert L.pot_gemm_workspace_bytes(2048, 10240, 8192, 3, 128) == 0
+    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 9 * 32 * 4096 * 4
 
 
 def test_status_strings(L):
