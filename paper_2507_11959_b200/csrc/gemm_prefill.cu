@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(PF_THREADS, PF_STAGES == 2 ? 2 : 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
                         __half* __restrict__ Y, float* __restrict__ partial, unsigned* __restrict__ counters,
-                        int* __restrict__ err) {
+                        int tiles_m, int n_full, int tail_splits, int* __restrict__ err) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -97,10 +97,28 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * (PF_BM * PF_MT), n0 = (int64_t)blockIdx.y * PF_BN;
+    // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
+    // into tail_splits items along K, so that the last, partly filled wave of CTAs is short.  Tiles are numbered
+    // with the token tile running fastest (CTAs that decode the same weight tile run together).
+    auto item = [&](int& tile, int& zsplit, int& splits) {
+        if ((int)blockIdx.x < n_full) {
+            tile = (int)blockIdx.x; zsplit = 0; splits = 1;
+        } else {
+            const int j = (int)blockIdx.x - n_full;
+            tile = n_full + j / tail_splits; zsplit = j % tail_splits; splits = tail_splits;
+        }
+    };
+    int64_t m0, n0, cb0, cb1;
+    {
+        int tile, zsplit, splits;
+        item(tile, zsplit, splits);
+        m0 = (int64_t)(tile % tiles_m) * (PF_BM * PF_MT);
+        n0 = (int64_t)(tile / tiles_m) * PF_BN;
+        // split item z of a tile owns column blocks [cb0, cb1), two stages each
+        cb0 = (int64_t)zsplit * (K / 128) / splits;
+        cb1 = ((int64_t)zsplit + 1) * (K / 128) / splits;
+    }
     const int64_t ncb = K / 128;
-    // split-K (few tiles, small M): CTA z of gridDim.z owns column blocks [cb0, cb1), two stages each
-    const int64_t cb0 = (int64_t)blockIdx.z * ncb / gridDim.z, cb1 = ((int64_t)blockIdx.z + 1) * ncb / gridDim.z;
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
@@ -243,7 +261,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
         const int mt = (warp - 2) >> 2;           // warps 2..5 read accumulator 0, warps 6..9 accumulator 1
         const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
-        const int splits = (int)gridDim.z;
+        int tile, zsplit, splits;  // recomputed here rather than kept in registers across the main loop
+        item(tile, zsplit, splits);
+        const int tail_index = tile - n_full;   // index of the tile among the split ones
+        const int64_t rows_alloc = M < PF_BM * PF_MT ? M : PF_BM * PF_MT;  // token rows kept per tile in the workspace
         auto store_row = [&](const uint32_t (&v)[32], int col) {  // 32 FP32 sums of one token -> FP16 -> Y
             __half* dst = Y + token * N + n0 + col;
             if (n0 + col + 32 <= N) {
@@ -271,12 +292,11 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (token < M) {
                 if (splits == 1) {
                     store_row(v, col);
-                } else {  // this split's partial sums, [split][token][feature] FP32 (N % 16 == 0: whole 16-byte pieces)
-                    float* dst = partial + ((int64_t)blockIdx.z * M + token) * N + n0 + col;
+                } else {  // this split's partial sums: [tail tile][split][token of the tile][128 features] FP32
+                    float* dst = partial + (((int64_t)tail_index * splits + zsplit) * rows_alloc + (token - m0)) * PF_BN + col;
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if (n0 + col + 4 * i < N)
-                            *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
             }
         }
@@ -286,35 +306,42 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             __shared__ unsigned s_prev;
             __threadfence();
             asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
-            const unsigned tile = blockIdx.y * gridDim.x + blockIdx.x;
-            if (threadIdx.x == 64) s_prev = atomicAdd(&counters[tile], 1u);
+            if (threadIdx.x == 64) s_prev = atomicAdd(&counters[tail_index], 1u);
             asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
             if (s_prev == (unsigned)splits - 1u) {
                 __threadfence();
-                if (token < M) {
-#pragma unroll 1
-                    for (int cc = 0; cc < PF_BN / 32; ++cc) {
-                        const int col = cc * 32;
-                        if (n0 + col >= N) break;
-                        float sum[32];
+                // The 256 epilogue threads walk the tile in 16-byte pieces, consecutive threads on consecutive
+                // pieces (coalesced), four pieces per thread in flight; the splits are added in ascending order.
+                const int pt = threadIdx.x - 64;
+                const float* tile0 = partial + (int64_t)tail_index * splits * rows_alloc * PF_BN;
+                const int64_t split_stride = rows_alloc * PF_BN;
+                const int npieces = (int)(rows_alloc * PF_BN / 4);
+                for (int p0 = pt; p0 < npieces; p0 += 4 * PF_PRODUCERS * 32) {
+                    float4 acc4[4];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) sum[i] = 0.f;
-                        for (int z = 0; z < splits; ++z) {
-                            const float* src = partial + ((int64_t)z * M + token) * N + n0 + col;
+                    for (int u = 0; u < 4; ++u) acc4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int z = 0; z < splits; ++z) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                if (n0 + col + 4 * i < N) {
-                                    const float4 t = __ldcg(reinterpret_cast<const float4*>(src + 4 * i));
-                                    sum[4 * i] += t.x; sum[4 * i + 1] += t.y; sum[4 * i + 2] += t.z; sum[4 * i + 3] += t.w;
-                                }
+                        for (int u = 0; u < 4; ++u) {
+                            const int pc = p0 + u * PF_PRODUCERS * 32;
+                            if (pc < npieces) {
+                                const float4 t = __ldcg(reinterpret_cast<const float4*>(tile0 + z * split_stride) + pc);
+                                acc4[u].x += t.x; acc4[u].y += t.y; acc4[u].z += t.z; acc4[u].w += t.w;
+                            }
                         }
-                        uint32_t v[32];
+                    }
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(sum[i]);
-                        store_row(v, col);
+                    for (int u = 0; u < 4; ++u) {
+                        const int pc = p0 + u * PF_PRODUCERS * 32;
+                        const int64_t row = m0 + pc / (PF_BN / 4), colx = n0 + 4 * (pc % (PF_BN / 4));
+                        if (pc < npieces && row < M && colx < N) {  // N % 16 == 0: a piece is inside or outside as a whole
+                            const __half2 h0 = __floats2half2_rn(acc4[u].x, acc4[u].y), h1 = __floats2half2_rn(acc4[u].z, acc4[u].w);
+                            *reinterpret_cast<uint2*>(Y + row * N + colx) =
+                                make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                        }
                     }
                 }
-                if (threadIdx.x == 64) counters[tile] = 0u;  // leave the workspace ready for the next call
+                if (threadIdx.x == 64) counters[tail_index] = 0u;  // leave the workspace ready for the next call
             }
         }
     }
@@ -349,36 +376,48 @@ bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group
     // TMA needs the X row pitch (2K bytes) to be a multiple of 16 -- implied by K % 128 == 0 -- and 32-bit box coordinates
     return M > 0 && N % 16 == 0 && K % 128 == 0 && M < (int64_t(1) << 31) && K < (int64_t(1) << 31);
 }
-// Split-K when the tiles cover less than half of the SMs (small M, narrow N): enough CTAs for two per SM, at least
-// four column blocks each.  (With more tiles than that the per-stage hand-off latency, which two co-resident
-// CTAs share, bounds the kernel either way and splitting only adds the reduction.)
-static int prefill_splits(int64_t M, int64_t N, int64_t K) {
-    const int64_t tiles = ((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)) * ((N + PF_BN - 1) / PF_BN);
-    if (2 * tiles > kSmCount) return 1;
-    int64_t s = 2 * kSmCount / tiles;
+// How the output tiles become work items.  Tiles run two CTAs per SM (296 slots); the tiles of the last, partly
+// filled wave -- or all tiles when they cover less than half of the SMs -- are cut along K into `splits` items
+// each (FP32 partial sums + an arrival counter per such tile in the workspace), at least four column blocks per item.
+struct PrefillPlan {
+    int tiles_m, tiles, n_full, n_tail, splits;
+    int64_t rows_alloc;
+    size_t counter_bytes, ws_bytes;
+};
+static PrefillPlan prefill_plan(int64_t M, int64_t N, int64_t K) {
+    PrefillPlan p{};
+    p.tiles_m = (int)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT));
+    p.tiles = p.tiles_m * (int)((N + PF_BN - 1) / PF_BN);
+    const int slots = 2 * kSmCount;
+    const int rem = p.tiles % slots;
+    int tail = 0;
+    if (2 * p.tiles <= kSmCount) tail = p.tiles;            // small problem: every tile is split
+    else if (p.tiles > slots && rem > 0 && 2 * rem <= slots) tail = rem;  // the last wave fills at most half of the slots
+    int64_t s = tail > 0 ? slots / tail : 1;
     const int64_t max_by_k = (K / 128) / 4;
     if (s > max_by_k) s = max_by_k;
+    if (s > 8 && tail != p.tiles) s = 8;
     if (s > 16) s = 16;
-    return s < 1 ? 1 : (int)s;
+    if (s < 2) { s = 1; tail = 0; }
+    p.splits = (int)s;
+    p.n_tail = tail;
+    p.n_full = p.tiles - tail;
+    p.rows_alloc = M < PF_BM * PF_MT ? M : PF_BM * PF_MT;
+    p.counter_bytes = tail ? ((size_t)tail * 4 + 255) / 256 * 256 : 0;
+    p.ws_bytes = tail ? p.counter_bytes + (size_t)tail * (size_t)s * (size_t)p.rows_alloc * PF_BN * 4 : 0;
+    return p;
 }
-static size_t prefill_counter_bytes(int64_t M, int64_t N) {
-    const int64_t tiles = ((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)) * ((N + PF_BN - 1) / PF_BN);
-    return ((size_t)tiles * 4 + 255) / 256 * 256;
-}
-// arrival counters (must start at zero; the kernel leaves them at zero) + [splits][M][N] FP32 partial sums
-size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) {
-    const int s = prefill_splits(M, N, K);
-    return s == 1 ? 0 : prefill_counter_bytes(M, N) + (size_t)s * (size_t)M * (size_t)N * 4;
-}
+// arrival counters (must start at zero; the kernel leaves them at zero) + FP32 partial sums of the split tiles
+size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) { return prefill_plan(M, N, K).ws_bytes; }
 
 static int* prefill_error_ptr();
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s) {
-    const int splits = prefill_splits(M, N, K);
-    if (splits > 1 && (!workspace || ws_bytes < gemm_prefill_workspace(M, N, K, bits, group))) return POT_ERR_WORKSPACE;
+    const PrefillPlan pl = prefill_plan(M, N, K);
+    if (pl.ws_bytes > 0 && (!workspace || ws_bytes < pl.ws_bytes)) return POT_ERR_WORKSPACE;
     unsigned* counters = (unsigned*)workspace;
-    float* partial = splits > 1 ? (float*)((char*)workspace + prefill_counter_bytes(M, N)) : nullptr;
+    float* partial = pl.ws_bytes > 0 ? (float*)((char*)workspace + pl.counter_bytes) : nullptr;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return POT_ERR_CUDA;
     CUtensorMap xmap;
@@ -390,15 +429,14 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
-    const dim3 grid((unsigned)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT)), (unsigned)((N + PF_BN - 1) / PF_BN), (unsigned)splits),
-        block(PF_THREADS);
+    const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits)), block(PF_THREADS);
     // too few CTAs to fill two per SM: one CTA per SM with the deeper pipeline
-    const bool deep = (int64_t)grid.x * grid.y * grid.z <= 2 * kSmCount && splits == 1;
+    const bool deep = (int64_t)grid.x <= 2 * kSmCount && pl.n_tail == 0;
     auto run = [&](auto kernel, int stages) -> pot_status_t {
         const size_t smem = pf_smem_bytes(stages);
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
-                          (__half*)Y, partial, counters, prefill_error_ptr());
+                          (__half*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
     if (deep) {
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4>, 4);

@@ -46,9 +46,12 @@ def test_size_helpers(L):
     ws = L.pot_gemv_workspace_bytes(4096, 11008, 3, 128)
     assert ws == 1024 + 256 * 22 * 16 * 4 and ws % 16 == 0
     assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
-    # M > 8 runs the tcgen05 kernel: no scratch unless few tiles make it split K (32 tiles -> 9 splits here)
-    assert L.pot_gemm_workspace_bytes(2048, 10240, 8192, 3, 128) == 0
-    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 9 * 32 * 4096 * 4
+    # M > 8 runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
+    # cover less than half of the SMs (32 tiles -> 9 splits of 32 token rows x 128 features), or those of a last
+    # wave that fills at most half of the 296 CTA slots (640 tiles -> 48 tail tiles x 6 splits x 256 rows).
+    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 32 * 9 * 32 * 128 * 4
+    assert L.pot_gemm_workspace_bytes(2048, 10240, 8192, 3, 128) == 256 + 48 * 6 * 256 * 128 * 4
+    assert L.pot_gemm_workspace_bytes(2048, 8192, 28672, 3, 128) == 0     # 512 tiles: the last wave is 73 % full
 
 
 def test_status_strings(L):
