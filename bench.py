@@ -183,9 +183,9 @@ def main():
         return torch.from_numpy(bits16.view(np.int16)).view(torch.float16).to(dev)
 
     # ---- build the chain: one layer of seeded weights, quantized on the device, replicated per layer
-    def build_chain(bits):
+    def build_chain(bits, projections=synth.LLAMA2_7B):
         protos = []
-        for i, pr in enumerate(synth.LLAMA2_7B):
+        for i, pr in enumerate(projections):
             W = f16(synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5"))
             packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
             tiled = B.pot_repack(packed, pr.K, bits, 0)
@@ -198,7 +198,7 @@ def main():
         layers = []
         for _ in range(args.layers):  # distinct buffers per layer: the chain streams from HBM
             layers.append([(pr, t.clone(), s.clone(), x, y, ws) for (pr, t, s, x, y, ws) in protos])
-        nbytes = args.layers * sum(gemv_bytes(pr.N, pr.K, bits, GROUP) for pr in synth.LLAMA2_7B)
+        nbytes = args.layers * sum(gemv_bytes(pr.N, pr.K, bits, GROUP) for pr in projections)
         return layers, nbytes
 
     def enqueue_chain(layers, bits, s):
@@ -395,6 +395,17 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
     ms2 = time_graph(g2, max(5, args.steps // 2), 3)
     ex["chain_2bit"] = {"GBps": bytes2 / ms2 / 1e6, "ms_per_step": ms2, "frac_of_measured_hbm": bytes2 / ms2 / 1e6 / hbm}
     del g2, layers2
+    torch.cuda.empty_cache()
+
+    # the same 3-bit chain with gate and up stored as one 4096 -> 22016 matrix (they share their input, as qkv do):
+    # 128 launches per step instead of 160 over the same weights
+    fused = (synth.LLAMA2_7B[0], synth.LLAMA2_7B[1], synth.Projection("gate_up", 4096, 22016), synth.LLAMA2_7B[4])
+    layersf, bytesf = build_chain(HEADLINE_BITS, fused)
+    gf = capture(lambda s: enqueue_chain(layersf, HEADLINE_BITS, s))
+    msf = time_graph(gf, max(5, args.steps // 2), 3)
+    ex["chain_3bit_gate_up_fused"] = {"GBps": bytesf / msf / 1e6, "ms_per_step": msf, "frac_of_measured_hbm": bytesf / msf / 1e6 / hbm,
+                                      "launches_per_step": 4 * args.layers}
+    del gf, layersf
     torch.cuda.empty_cache()
 
     def rotating(make, copies):
