@@ -97,9 +97,9 @@ extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t
     if (N % 16 != 0) return POT_ERR_SHAPE;
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
     if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-    if (bits == 2) return launch_gemv_mma<2>(packed, scales, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    if (bits == 3) return launch_gemv_mma<3>(packed, scales, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    return launch_gemv_mma<4>(packed, scales, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    if (bits == 2) return launch_gemv_mma<2>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    if (bits == 3) return launch_gemv_mma<3>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    return launch_gemv_mma<4>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
 }
 
 extern "C" pot_status_t pot_gemv_host(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -139,9 +139,10 @@ extern "C" pot_status_t uint_gemv(const void* packed, const void* scales, const 
     if (N % 16 != 0) return POT_ERR_SHAPE;
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
     if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-    if (bits == 2) return launch_ring<2, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
-    if (bits == 3) return launch_ring<3, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
-    return launch_ring<4, RG_UINT_FMA, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, ring_error_ptr(), s);
+    // same kernel as pot_gemv (tensor-core path); only the decode differs
+    if (bits == 2) return launch_gemv_mma<2, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    if (bits == 3) return launch_gemv_mma<3, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    return launch_gemv_mma<4, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
 }
 
 // ------------------------------------------------------------------------------------------

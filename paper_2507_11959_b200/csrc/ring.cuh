@@ -30,13 +30,13 @@ namespace pot {
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 
-enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3, RG_POT_MMA1W = 4 };
+enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3, RG_POT_MMA1W = 4, RG_UINT_MMA1 = 5, RG_UINT_MMA1W = 6 };
 
 constexpr int RG_Q = 5;  // steps per ring slot (one bulk copy) = warps per consumer group
 // Consumer groups per CTA: slot m is consumed by group m % groups, warp i of it takes step i.  The tensor-core
 // GEMV needs fewer registers per thread, so one more group of warps fits (RG_POT_MMA1W); whether that pays
 // depends on how evenly the CTA's steps divide among the warps, see launch_gemv_mma.
-__host__ __device__ constexpr int rg_groups(int mode) { return mode == RG_POT_MMA1W ? 4 : 3; }
+__host__ __device__ constexpr int rg_groups(int mode) { return (mode == RG_POT_MMA1W || mode == RG_UINT_MMA1W) ? 4 : 3; }
 __host__ __device__ constexpr int rg_consumers(int mode) { return rg_groups(mode) * RG_Q; }
 __host__ __device__ constexpr int rg_threads(int mode) { return (rg_consumers(mode) + 1) * 32; }
 __host__ __device__ constexpr int rg_unit_bytes(int bits) { return 256 * bits; }
@@ -197,9 +197,10 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     constexpr bool XSMEM = (XMODE != 0);
     constexpr bool XWIDE = (XMODE == 2);
     constexpr bool MMA = (MODE == RG_POT_MMA);
-    constexpr bool UNIFORM = (MODE == RG_UINT_FMA);
+    constexpr bool UNIFORM_TC = (MODE == RG_UINT_MMA1 || MODE == RG_UINT_MMA1W);  // the twin on the tensor-core path
+    constexpr bool UNIFORM = (MODE == RG_UINT_FMA) || UNIFORM_TC;
     constexpr int RG_CONSUMERS = rg_consumers(MODE), RG_GROUPS = rg_groups(MODE);
-    constexpr bool MMA1 = (MODE == RG_POT_MMA1 || MODE == RG_POT_MMA1W);
+    constexpr bool MMA1 = (MODE == RG_POT_MMA1 || MODE == RG_POT_MMA1W) || UNIFORM_TC;
     constexpr bool TC = MMA || MMA1;  // tensor-core modes: lane (gid, tig) owns quarter tig of rows gid and gid + 8
     static_assert(!MMA || MT == 1, "one tile of eight tokens");
     constexpr int TOK = MMA ? 8 * MT : 1;
@@ -266,10 +267,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     // scales (and zero-points) of a step are fetched one step ahead, straight from global memory.  The
     // buffers keep the raw 16-bit loads: any arithmetic on them here would make the warp wait for the load.
     // tensor-core modes: the scale of this lane's quarter, for both rows and the four units of a step
-    uint32_t sc1[2][TC ? 8 : 1];
+    uint32_t sc1[2][TC ? 8 : 1], zp1[2][UNIFORM_TC ? 8 : 1];
     auto load_scales_mma1 = [&](int64_t rb, int c, int buf) {
         // one 64-bit address per step; the eight loads use constant offsets from it
-        const uint16_t* s0 = scales + (rb * 16 + gid) * gpr + (int64_t)c * (4 * spg) + (spg == 2 ? (tig >> 1) : 0);
+        const int64_t so = (rb * 16 + gid) * gpr + (int64_t)c * (4 * spg) + (spg == 2 ? (tig >> 1) : 0);
+        const uint16_t* s0 = scales + so;
         const int64_t up = 8 * (int64_t)gpr;
         const int nu = (int)(ncb - 4 * (int64_t)c);  // units of this step (>= 4 except at the ragged end of a row)
 #pragma unroll
@@ -279,6 +281,11 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                 uint32_t v = 0x3C00u;
                 if (u < nu) v = (uint32_t)__ldg(s0 + (h ? up : 0) + (spg == 2 ? 2 * u : u));
                 sc1[buf][h * 4 + u] = v;
+                if constexpr (UNIFORM_TC) {
+                    uint32_t z = 0u;
+                    if (u < nu) z = (uint32_t)__ldg(zeros + so + (h ? up : 0) + (spg == 2 ? 2 * u : u));
+                    zp1[buf][h * 4 + u] = z;
+                }
             }
     };
     uint32_t sc[2][2][2], zp[2][2][2];
@@ -378,8 +385,16 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             int c_s = c - wig;
             while (c_s < 0) { c_s += spr; --rb_s; }
             const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - (rb_s * ncb + 4 * (int64_t)c_s);
-            // plane k of a unit holds word k of every (row, quarter): this lane's word sits at byte 4 * lane
-            const unsigned char* ubase = ring + (size_t)slot * SLOT + uoff * UB + lane * 4;
+            // PoT: plane k of a unit holds word k of every (row, quarter): this lane's word sits at byte 4 * lane.
+            // Uniform twin: the quarter's words sit at record words 2*tig, 2*tig+1 (n = 2), 2*tig, 2*tig+1, 8+tig
+            // (n = 3) or 4*tig .. 4*tig+3 (n = 4); record word w is byte (w / 4) * 256 + row * 16 + (w % 4) * 4.
+            const unsigned char* ubase = ring + (size_t)slot * SLOT + uoff * UB + (UNIFORM_TC ? gid * 16 : lane * 4);
+            int woff[BITS];
+#pragma unroll
+            for (int k = 0; k < BITS; ++k) {
+                const int w = BITS == 4 ? 4 * tig + k : (k < 2 ? 2 * tig + k : 8 + tig);
+                woff[k] = UNIFORM_TC ? (w >> 2) * 256 + (w & 3) * 4 : k * 256;
+            }
             float acc1[2][4];
 #pragma unroll
             for (int i = 0; i < 2; ++i)
@@ -398,7 +413,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                         for (int k = 0; k < BITS; ++k) {
                             wreg[u][h][k] = 0u;
                             if (4 * (int64_t)c + u < ncb)
-                                wreg[u][h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
+                                wreg[u][h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + woff[k] + h * 128);
                         }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
@@ -413,7 +428,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
 #pragma unroll
                         for (int k = 0; k < BITS; ++k) {
                             if constexpr (RELEASE_EARLY) w[h][k] = wreg[u][h][k];
-                            else w[h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + k * 256 + h * 128);
+                            else w[h][k] = *reinterpret_cast<const uint32_t*>(ubase + u * UB + woff[k] + h * 128);
                         }
                     uint32_t xq[16];  // 32 activations of quarter tig (of token gid): the B fragments of eight MMAs
                     if constexpr (MMA1) {
@@ -435,8 +450,29 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                         }
                     }
                     uint32_t lo[16], hi[16];
-                    potl::pot_decode32<BITS, 1>(w[0], 0, sc1[buf][u] * 0x10001u, lo);
-                    potl::pot_decode32<BITS, 1>(w[1], 0, sc1[buf][4 + u] * 0x10001u, hi);
+                    if constexpr (UNIFORM_TC) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            // the quarter's words, placed where uint_decode_pairs16 looks for blocks 0 and 1
+                            uint32_t q[BITS == 3 ? 9 : BITS];
+#pragma unroll
+                            for (int k = 0; k < BITS; ++k) q[(BITS == 3 && k == 2) ? 8 : k] = w[h][k];
+                            potl::UintParams pr;
+                            pr.s2 = potl::bits_h2(sc1[buf][h * 4 + u] * 0x10001u);
+                            pr.z = potl::bits_h2(zp1[buf][h * 4 + u] * 0x10001u);
+                            uint32_t a8[8], b8[8];
+                            potl::uint_decode_pairs16<BITS>(q, 0, pr, a8);
+                            potl::uint_decode_pairs16<BITS>(q, 1, pr, b8);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                (h ? hi : lo)[i] = a8[i];
+                                (h ? hi : lo)[8 + i] = b8[i];
+                            }
+                        }
+                    } else {
+                        potl::pot_decode32<BITS, 1>(w[0], 0, sc1[buf][u] * 0x10001u, lo);
+                        potl::pot_decode32<BITS, 1>(w[1], 0, sc1[buf][4 + u] * 0x10001u, hi);
+                    }
 #pragma unroll
                     for (int j = 0; j < 8; ++j)  // two accumulators: half the length of the dependent chain
                         rg_mma(acc1[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
@@ -632,14 +668,15 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
 
 // GEMV on the warp-level tensor-core path with 15 or 20 consumer warps: a warp works through whole steps, so the
 // time is (steps per warp, rounded up) x (time per step, about 1.2 x longer when 20 warps share the SM).
-template <int BITS>
-pot_status_t launch_gemv_mma(const void* packed, const void* scales, int64_t N, int64_t K, int group, const void* x, void* y,
-                             void* workspace, int* err, cudaStream_t s) {
+template <int BITS, bool UNIFORM_CODES = false>
+pot_status_t launch_gemv_mma(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
+                             const void* x, void* y, void* workspace, int* err, cudaStream_t s) {
     const RingPlan p = plan_ring(N, K, 1, BITS, 1, false, 3);
     const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
     const double t3 = (double)((per_cta + 14) / 15), t4 = 1.2 * (double)((per_cta + 19) / 20);
-    if (t4 < t3) return launch_ring<BITS, RG_POT_MMA1W, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, err, s);
-    return launch_ring<BITS, RG_POT_MMA1, 1>(packed, scales, nullptr, N, K, group, x, 1, y, workspace, err, s);
+    constexpr int NARROW = UNIFORM_CODES ? RG_UINT_MMA1 : RG_POT_MMA1, WIDE = UNIFORM_CODES ? RG_UINT_MMA1W : RG_POT_MMA1W;
+    if (t4 < t3) return launch_ring<BITS, WIDE, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s);
+    return launch_ring<BITS, NARROW, 1>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s);
 }
 
 }  // namespace pot
