@@ -20,6 +20,20 @@
 
 namespace pot {
 
+// two FP16 x FP16 products accumulated in FP32 (mixed-precision FMA: no conversion instructions)
+__device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
+    asm("{\n\t"
+        ".reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %2;\n\t"
+        "mov.b32 {xl, xh}, %3;\n\t"
+        "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
+        "fma.rn.f32.f16 %1, wh, xh, %1;\n\t"
+        "}"
+        : "+f"(acc0), "+f"(acc1)
+        : "r"(w2), "r"(x2));
+}
+
+
 // ------------------------------------------------------------------------------------------
 // canonical layout, one warp per row
 // ------------------------------------------------------------------------------------------

@@ -1,15 +1,15 @@
-// Ring-buffered streaming kernel for the decode GEMV (CUDA cores) and the small-batch GEMM (tensor
-// cores) on the tiled layout.
+// Ring-buffered streaming kernel for the decode GEMV (PoT and the uniform twin) and the small-batch
+// GEMM on the tiled layout; the multiply-accumulate runs on warp-level tensor-core MMAs.
 //
 // One persistent CTA per SM.  A producer warp streams the CTA's share of the packed codes from
 // HBM into a shared-memory ring with 1-D bulk copies (cp.async.bulk + mbarrier transaction
 // counts), several steps (up to 20 KB) per copy since the share is one contiguous byte range in the
 // tiled layout; the bytes in flight therefore cost no registers, and the whole share of a short
 // matrix can be requested before the first byte arrives.  Consumer warps take the ring stages
-// round-robin, pull their records out of shared memory with conflict-free 16-byte loads, decode
+// round-robin, pull their share of the records out of shared memory (one word per lane and plane), decode
 // them in registers (integer mask / shift-add into the scale's bit pattern) and accumulate in
-// FP32 -- with the mixed-precision FMA (GEMV) or with warp-level MMAs whose A fragment is the
-// decoded weights (small batch).
+// FP32 with warp-level MMAs whose A fragment is the decoded weights (B = the activation vector in
+// every column for the GEMV, one token per column for the small batch).
 //
 // Work decomposition: the matrix is a sequence of steps; step g = 16 rows x 512 columns
 // (row block g / spr, columns 512 * (g % spr)).  CTA b owns the contiguous range
@@ -30,7 +30,7 @@ namespace pot {
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 
-enum RingMode { RG_POT_FMA = 0, RG_UINT_FMA = 1, RG_POT_MMA = 2, RG_POT_MMA1 = 3, RG_POT_MMA1W = 4, RG_UINT_MMA1 = 5, RG_UINT_MMA1W = 6 };
+enum RingMode { RG_POT_MMA = 2, RG_POT_MMA1 = 3, RG_POT_MMA1W = 4, RG_UINT_MMA1 = 5, RG_UINT_MMA1W = 6 };
 
 constexpr int RG_Q = 5;  // steps per ring slot (one bulk copy) = warps per consumer group
 // Consumer groups per CTA: slot m is consumed by group m % groups, warp i of it takes step i.  The tensor-core
@@ -48,7 +48,6 @@ struct RingPlan {
     int64_t total_steps;
     int stages;
     bool x_in_smem;
-    bool x_wide;         // GEMV only: x staged one FP16 value per 32-bit word (no half2 unpacking in the loop)
     size_t x_bytes;      // shared-memory bytes for the staged activations (0 if read from global)
     size_t cmb_bytes;    // shared-memory bytes for combining the steps of a row block inside the CTA (0 = off)
     size_t smem_bytes;   // total dynamic shared memory
@@ -56,15 +55,14 @@ struct RingPlan {
     size_t ws_bytes;
 };
 
-inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, bool wide_ok = true, int groups = 3) {
+inline RingPlan plan_ring(int64_t N, int64_t K, int64_t M, int bits, int tok, int groups = 3) {
     RingPlan p;
     const int64_t nrb = N / 16, ncb = K / 128;
     p.spr = (int)((ncb + 3) / 4);
     p.total_steps = nrb * p.spr;
     p.grid = (int)(p.total_steps < kSmCount ? p.total_steps : kSmCount);
-    p.x_wide = wide_ok && (tok == 1) && (size_t)K * 4 <= 48 * 1024;
     // the small-batch mode stages a full tile of eight tokens (fragment order), whatever M is
-    const size_t xb = (size_t)(tok > 1 ? tok : M) * (size_t)K * (p.x_wide ? 4 : 2);
+    const size_t xb = (size_t)(tok > 1 ? tok : M) * (size_t)K * 2;
     p.x_in_smem = xb <= (tok > 1 ? 96 : 64) * 1024;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
     const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
@@ -150,30 +148,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 template <int NC>
 __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NC * 32) : "memory"); }
 
-__device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
-    asm("{\n\t"
-        ".reg .b16 wl, wh, xl, xh;\n\t"
-        "mov.b32 {wl, wh}, %2;\n\t"
-        "mov.b32 {xl, xh}, %3;\n\t"
-        "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
-        "fma.rn.f32.f16 %1, wh, xh, %1;\n\t"
-        "}"
-        : "+f"(acc0), "+f"(acc1)
-        : "r"(w2), "r"(x2));
-}
-// same with x already split: x0 / x1 hold one FP16 value each in their low 16 bits
-__device__ __forceinline__ void rg_fma2_wide(float& acc0, float& acc1, uint32_t w2, uint32_t x0, uint32_t x1) {
-    asm("{\n\t"
-        ".reg .b16 wl, wh, xa, xb, d0, d1;\n\t"
-        "mov.b32 {wl, wh}, %2;\n\t"
-        "mov.b32 {xa, d0}, %3;\n\t"
-        "mov.b32 {xb, d1}, %4;\n\t"
-        "fma.rn.f32.f16 %0, wl, xa, %0;\n\t"
-        "fma.rn.f32.f16 %1, wh, xb, %1;\n\t"
-        "}"
-        : "+f"(acc0), "+f"(acc1)
-        : "r"(w2), "r"(x0), "r"(x1));
-}
 __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
     asm volatile(
@@ -182,26 +156,22 @@ __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// MODE RG_POT_FMA / RG_UINT_FMA / RG_POT_MMA1: M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
+// MODE RG_POT_MMA1(W) / RG_UINT_MMA1(W): M = 1.  MODE RG_POT_MMA: M <= 8*MT tokens.
 // RG_POT_MMA1 is the GEMV on the warp-level tensor-core path: the activation vector fills every column of the
 // MMA's B operand, lane (gid, tig) owns quarter tig of the records of rows gid and gid + 8 -- exactly its share
 // of the A fragment -- and the MMA adds up the four quarters, so there is no cross-lane reduction and the
 // multiply-accumulate costs one instruction per 256 weights instead of one per weight.
-template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = staged packed, 2 = staged wide
+template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = x staged in shared memory
 __global__ void __launch_bounds__(rg_threads(MODE), 1)
 ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
             int64_t N, int64_t K, int G, int spr, int64_t total_steps, int stages, int x_bytes, int cmb_bytes,
             const __half* __restrict__ X, int M, __half* __restrict__ Y, float* __restrict__ partial,
             unsigned* __restrict__ counters, int* __restrict__ err) {
-    constexpr int NW = 4 * BITS;
     constexpr bool XSMEM = (XMODE != 0);
-    constexpr bool XWIDE = (XMODE == 2);
     constexpr bool MMA = (MODE == RG_POT_MMA);
     constexpr bool UNIFORM_TC = (MODE == RG_UINT_MMA1 || MODE == RG_UINT_MMA1W);  // the twin on the tensor-core path
-    constexpr bool UNIFORM = (MODE == RG_UINT_FMA) || UNIFORM_TC;
     constexpr int RG_CONSUMERS = rg_consumers(MODE), RG_GROUPS = rg_groups(MODE);
     constexpr bool MMA1 = (MODE == RG_POT_MMA1 || MODE == RG_POT_MMA1W) || UNIFORM_TC;
-    constexpr bool TC = MMA || MMA1;  // tensor-core modes: lane (gid, tig) owns quarter tig of rows gid and gid + 8
     static_assert(!MMA || MT == 1, "one tile of eight tokens");
     constexpr int TOK = MMA ? 8 * MT : 1;
     constexpr int SLOT = rg_slot_bytes(BITS);
@@ -259,16 +229,15 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     }
 
     // -------------------- consumers --------------------------------------------------------------------
-    const int gid = TC ? (lane >> 2) : (lane & 7);
-    const int tig = TC ? (lane & 3) : (lane >> 3);
+    const int gid = lane >> 2, tig = lane & 3;  // MMA fragment coordinates: rows gid and gid + 8, quarter tig
     const int gpr = (int)(K / G);
     const int spg = 128 / G;
 
     // scales (and zero-points) of a step are fetched one step ahead, straight from global memory.  The
     // buffers keep the raw 16-bit loads: any arithmetic on them here would make the warp wait for the load.
-    // tensor-core modes: the scale of this lane's quarter, for both rows and the four units of a step
-    uint32_t sc1[2][TC ? 8 : 1], zp1[2][UNIFORM_TC ? 8 : 1];
-    auto load_scales_mma1 = [&](int64_t rb, int c, int buf) {
+    // sc1 / zp1: the scale (zero-point) of this lane's quarter, for both rows and the four units of a step
+    uint32_t sc1[2][8], zp1[2][UNIFORM_TC ? 8 : 1];
+    auto load_scales = [&](int64_t rb, int c, int buf) {
         // one 64-bit address per step; the eight loads use constant offsets from it
         const int64_t so = (rb * 16 + gid) * gpr + (int64_t)c * (4 * spg) + (spg == 2 ? (tig >> 1) : 0);
         const uint16_t* s0 = scales + so;
@@ -287,25 +256,6 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                     zp1[buf][h * 4 + u] = z;
                 }
             }
-    };
-    uint32_t sc[2][2][2], zp[2][2][2];
-    auto load_scales = [&](int64_t rb, int c, int buf) {
-        if constexpr (TC) { load_scales_mma1(rb, c, buf); return; }
-        const int64_t cb = 4 * (int64_t)c + tig;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            sc[buf][h][0] = sc[buf][h][1] = 0x3C00u;
-            zp[buf][h][0] = zp[buf][h][1] = 0u;
-            if (cb < ncb) {
-                const int64_t so = (rb * 16 + gid + 8 * h) * gpr + cb * spg;
-                sc[buf][h][0] = (uint32_t)__ldg(scales + so);
-                sc[buf][h][1] = (uint32_t)__ldg(scales + so + spg - 1);
-                if constexpr (UNIFORM) {
-                    zp[buf][h][0] = (uint32_t)__ldg(zeros + so);
-                    zp[buf][h][1] = (uint32_t)__ldg(zeros + so + spg - 1);
-                }
-            }
-        }
     };
     // Slot (bulk copy) m holds steps m*Q .. m*Q+Q-1 and belongs to warp group m % GROUPS; warp i of the group
     // takes step m*Q + i.  A warp therefore meets the barriers of "its" slots once per fill and in order,
@@ -345,16 +295,9 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
             const int n16 = (int)(K / 8);
             for (int i = threadIdx.x; i < n16; i += RG_CONSUMERS * 32) {
                 const uint4 v = __ldg(src + i);
-                if constexpr (XWIDE) {
-                    dst[2 * i] = make_uint4(v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16);
-                    dst[2 * i + 1] = make_uint4(v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16);
-                } else if constexpr (MMA1) {
-                    // chunk (quarter t, part j) of a unit goes to position j * 4 + t: the four lanes tig = 0..3 then
-                    // read 64 contiguous bytes
-                    dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v;
-                } else {
-                    dst[i] = v;
-                }
+                // chunk (quarter t, part j) of a unit goes to position j * 4 + t: the four lanes tig = 0..3 then read
+                // 64 contiguous bytes
+                dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v;
             }
         }
         consumer_bar_sync<RG_CONSUMERS>();
@@ -372,14 +315,12 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         int c_next = c + J_STRIDE;
         while (c_next >= spr) { c_next -= spr; ++rb_next; }
         if (j + J_STRIDE < nsteps) load_scales(rb_next, c_next, buf ^ 1);
-        const int64_t cb = 4 * (int64_t)c + tig;
-        const bool valid = cb < ncb;
         if (!mbar_wait(smem_u32(&bars[slot]), phase)) {
             if (err && lane == 0) atomicCAS(err, 0, 2 | (m << 8) | (warp << 16) | (j << 24));
         }
-        float r0 = 0.f, r1 = 0.f;  // RG_POT_MMA1: the sums of rows gid and gid + 8
+        float r0 = 0.f, r1 = 0.f;  // GEMV: the sums of rows gid and gid + 8
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        if constexpr (TC) {
+        {
             // units between the slot's first step (wig steps back) and this one, without divisions
             int64_t rb_s = rb;
             int c_s = c - wig;
@@ -487,65 +428,6 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[e] = acc1[0][e] + acc1[1][e];
         }
-        if constexpr (!TC) {
-        uint32_t rec[2][NW];
-        {
-            // records are fetched with lane (column block, row) = (lane / 8, lane % 8): 8 lanes read 128
-            // contiguous bytes, free of bank conflicts
-            const int ftig = lane >> 3, fgid = lane & 7;
-            // units between the slot's first step (wig steps back) and this one, without divisions
-            int64_t rb_s = rb;
-            int c_s = c - wig;
-            while (c_s < 0) { c_s += spr; --rb_s; }
-            const int64_t uoff = (rb * ncb + 4 * (int64_t)c) - (rb_s * ncb + 4 * (int64_t)c_s) + ftig;
-            const bool fvalid = 4 * (int64_t)c + ftig < ncb;
-            const uint4* unit = reinterpret_cast<const uint4*>(ring + (size_t)slot * SLOT + uoff * UB);
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int t = 0; t < BITS; ++t) {
-                    uint4 q = make_uint4(0, 0, 0, 0);
-                    if (fvalid) q = unit[t * 16 + fgid + 8 * h];
-                    rec[h][4 * t + 0] = q.x; rec[h][4 * t + 1] = q.y; rec[h][4 * t + 2] = q.z; rec[h][4 * t + 3] = q.w;
-                }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars[stages + slot]));  // one step of the slot is consumed
-
-        {
-            if (valid) {
-#pragma unroll
-                for (int T = 0; T < 4; ++T) {
-                    uint32_t xw[XWIDE ? 32 : 16];
-#pragma unroll
-                    for (int i = 0; i < (XWIDE ? 8 : 4); ++i) {
-                        const uint4 v = XWIDE ? xs[cb * 32 + 8 * T + i]
-                                              : (XSMEM ? xs[cb * 16 + 4 * T + i]
-                                                       : __ldg(reinterpret_cast<const uint4*>(X) + cb * 16 + 4 * T + i));
-                        xw[4 * i + 0] = v.x; xw[4 * i + 1] = v.y; xw[4 * i + 2] = v.z; xw[4 * i + 3] = v.w;
-                    }
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t w2[16];
-                        if constexpr (!UNIFORM) {
-                            potl::pot_decode32<BITS>(rec[h], T, sc[buf][h][T >> 1] * 0x10001u, w2);
-                        } else {
-                            potl::UintParams pr;
-                            pr.s2 = potl::bits_h2(sc[buf][h][T >> 1] * 0x10001u);
-                            pr.z = potl::bits_h2(zp[buf][h][T >> 1] * 0x10001u);
-                            potl::uint_decode32<BITS>(rec[h], T, pr, w2);
-                        }
-#pragma unroll
-                        for (int p = 0; p < 16; ++p) {
-                            if constexpr (XWIDE) rg_fma2_wide(acc[2 * h], acc[2 * h + 1], w2[p], xw[2 * p], xw[2 * p + 1]);
-                            else rg_fma2(acc[2 * h], acc[2 * h + 1], w2[p], xw[p]);
-                        }
-                    }
-                }
-            }
-        }
-
-        }
         // ---- deliver the step's partial sums -----------------------------------------------------------
         // spr == 1: the step is the whole row block, write Y.  Otherwise the 16*TOK sums go to a slot:
         // in shared memory when every step of the row block belongs to this CTA (the common case),
@@ -557,11 +439,6 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                             : (local ? cmb + (size_t)(rb_g0 - g_begin + c) * (16 * TOK)
                                      : partial + (rb_g0 + c) * (16 * TOK));
         if (!MMA) {
-            if constexpr (!MMA1) {
-                r0 = acc[0] + acc[1], r1 = acc[2] + acc[3];
-                r0 += __shfl_xor_sync(0xffffffffu, r0, 8); r0 += __shfl_xor_sync(0xffffffffu, r0, 16);
-                r1 += __shfl_xor_sync(0xffffffffu, r1, 8); r1 += __shfl_xor_sync(0xffffffffu, r1, 16);
-            }
             if (tig == 0) {
                 if (whole) {
                     Y[rb * 16 + gid] = __float2half_rn(r0);
@@ -649,8 +526,7 @@ inline int ring_error_fetch() {
 template <int BITS, int MODE, int MT>
 pot_status_t launch_ring(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                          const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
-    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, MODE == RG_POT_FMA || MODE == RG_UINT_FMA,
-                                 rg_groups(MODE));
+    const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, rg_groups(MODE));
     auto run = [&](auto kernel) -> pot_status_t {
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         unsigned* counters = (unsigned*)workspace;
@@ -659,9 +535,6 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
                           (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
                           (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
     };
-    if constexpr (MODE == RG_POT_FMA || MODE == RG_UINT_FMA) {
-        if (p.x_in_smem && p.x_wide) return run(ring_kernel<BITS, MODE, MT, 2>);
-    }
     if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, 1>);
     return run(ring_kernel<BITS, MODE, MT, 0>);
 }
@@ -671,7 +544,7 @@ pot_status_t launch_ring(const void* packed, const void* scales, const void* zer
 template <int BITS, bool UNIFORM_CODES = false>
 pot_status_t launch_gemv_mma(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                              const void* x, void* y, void* workspace, int* err, cudaStream_t s) {
-    const RingPlan p = plan_ring(N, K, 1, BITS, 1, false, 3);
+    const RingPlan p = plan_ring(N, K, 1, BITS, 1, 3);
     const int64_t per_cta = (p.total_steps + p.grid - 1) / p.grid;
     const double t3 = (double)((per_cta + 14) / 15), t4 = 1.2 * (double)((per_cta + 19) / 20);
     constexpr int NARROW = UNIFORM_CODES ? RG_UINT_MMA1 : RG_POT_MMA1, WIDE = UNIFORM_CODES ? RG_UINT_MMA1W : RG_POT_MMA1W;
