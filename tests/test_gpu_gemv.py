@@ -120,3 +120,21 @@ def test_pot_gemm_fallback_matches_oracle(B, oracle, bits, M):
         Yg = B.pot_gemm(c.d_packed, c.d_S, K, bits, G, f16_dev(X), B.CANONICAL)
         ok, worst, tight = gate(bits_of(Yg), Y, A)
         assert ok and tight < 4.0, ("fallback", N, K, M, worst, tight)
+
+
+def test_gemv_with_activations_too_long_for_shared_memory(B, oracle):
+    """K = 33024: the activation vector (66 KB) no longer fits the kernel's shared-memory staging area and is read
+    from global memory instead -- PoT and uniform twin."""
+    bits, G, N, K = 3, 128, 32, 33024
+    X = acts(1, K, 900)
+    c = PotCase(N, K, bits, G, dist="t5", seed=(4, 900))
+    Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
+    y = B.pot_gemv(c.tiled(), c.d_S, K, bits, G, f16_dev(X[0]), B.TILED)
+    ok, worst, tight = gate(bits_of(y), Y[0], A[0])
+    assert ok and tight < 4.0, ("pot", worst, tight)
+    u = UintCase(N, K, bits, G, dist="t5", seed=(4, 901))
+    Y, A = oracle.uint_matmul(u.packed, u.S, u.Z, K, bits, G, X)
+    y = B.uint_gemv(u.tiled(), u.d_S, u.d_Z, K, bits, G, f16_dev(X[0]), B.TILED)
+    ok, worst, tight = gate(bits_of(y), Y[0], A[0])
+    assert ok and tight < 4.0, ("uint", worst, tight)
+    assert B.pot_debug_errors() == (0, 0, 0)
