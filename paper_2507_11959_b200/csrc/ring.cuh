@@ -161,12 +161,42 @@ __device__ __forceinline__ void rg_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
 // MMA's B operand, lane (gid, tig) owns quarter tig of the records of rows gid and gid + 8 -- exactly its share
 // of the A fragment -- and the MMA adds up the four quarters, so there is no cross-lane reduction and the
 // multiply-accumulate costs one instruction per 256 weights instead of one per weight.
-template <int BITS, int MODE, int MT, int XMODE>  // XMODE: 0 = x from global, 1 = x staged in shared memory
-__global__ void __launch_bounds__(rg_threads(MODE), 1)
-ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros,
-            int64_t N, int64_t K, int G, int spr, int64_t total_steps, int stages, int x_bytes, int cmb_bytes,
-            const __half* __restrict__ X, int M, __half* __restrict__ Y, float* __restrict__ partial,
-            unsigned* __restrict__ counters, int* __restrict__ err) {
+struct RingArgs {
+    const uint4* packed;
+    const uint16_t* scales;
+    const uint16_t* zeros;
+    int64_t N, K;
+    int G, spr;
+    int64_t total_steps;
+    int stages, x_bytes, cmb_bytes;
+    const __half* X;
+    int M;
+    __half* Y;
+    float* partial;
+    unsigned* counters;
+};
+
+__device__ __forceinline__ void mbar_inval(uint32_t bar) { asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory"); }
+
+// One GEMV / small-batch GEMM, executed by the whole CTA.  CHAIN = false: the body of a stand-alone launch (chained
+// to its neighbours in the stream by programmatic dependent launch).  CHAIN = true: operation `op` of a persistent
+// kernel that runs a list of dependent operations; `sync` is its grid-wide arrival counter: every CTA arrives when
+// it has delivered its part of an operation, and the consumers of the next operation wait for all CTAs before
+// they touch the activations (the producer warp does not wait: the weights are constants, it streams ahead).
+template <int BITS, int MODE, int MT, int XMODE, bool CHAIN>  // XMODE: 0 = x from global, 1 = x staged in shared memory
+__device__ __forceinline__ void ring_body(const RingArgs& ra, int* __restrict__ err, unsigned* sync, int op, int prev_stages) {
+    const uint4* __restrict__ packed = ra.packed;
+    const uint16_t* __restrict__ scales = ra.scales;
+    const uint16_t* __restrict__ zeros = ra.zeros;
+    const int64_t N = ra.N, K = ra.K;
+    const int G = ra.G, spr = ra.spr;
+    const int64_t total_steps = ra.total_steps;
+    const int stages = ra.stages, x_bytes = ra.x_bytes, cmb_bytes = ra.cmb_bytes;
+    const __half* __restrict__ X = ra.X;
+    const int M = ra.M;
+    __half* __restrict__ Y = ra.Y;
+    float* __restrict__ partial = ra.partial;
+    unsigned* __restrict__ counters = ra.counters;
     constexpr bool XSMEM = (XMODE != 0);
     constexpr bool MMA = (MODE == RG_POT_MMA);
     constexpr bool UNIFORM_TC = (MODE == RG_UINT_MMA1 || MODE == RG_UINT_MMA1W);  // the twin on the tensor-core path
@@ -194,6 +224,10 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         return (int64_t)rbq * ncb + 4 * (int64_t)((uint32_t)g - rbq * (uint32_t)spr);
     };
 
+    if constexpr (CHAIN) {  // the previous operation's barriers (another ring length) make room first
+        if ((int)threadIdx.x < 2 * prev_stages) mbar_inval(smem_u32(&bars[threadIdx.x]));
+        __syncthreads();
+    }
     if (threadIdx.x < stages) {  // one thread per ring slot
         mbar_init(smem_u32(&bars[threadIdx.x]), 1);                // full: the producer's expect_tx arrival
         mbar_init(smem_u32(&bars[stages + threadIdx.x]), RG_Q);    // empty: one arrival per consumed step
@@ -204,7 +238,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         for (int i = threadIdx.x; i < nsteps / spr + 3; i += blockDim.x) cmb_cnt[i] = 0u;
     }
     __syncthreads();
-    pdl_launch_dependents();
+    if constexpr (!CHAIN) pdl_launch_dependents();
 
     if (warp == RG_CONSUMERS) {
         // ---------------- producer: weights do not depend on the previous kernel, start at once ----------
@@ -225,9 +259,7 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
                 bulk_g2s(smem_u32(ring + (size_t)slot * SLOT), packed + u0 * (16 * BITS), bytes, full);
             }
         }
-        return;
-    }
-
+    } else {
     // -------------------- consumers --------------------------------------------------------------------
     const int gid = lane >> 2, tig = lane & 3;  // MMA fragment coordinates: rows gid and gid + 8, quarter tig
     const int gpr = (int)(K / G);
@@ -269,7 +301,22 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
     while (c >= spr) { c -= spr; ++rb; }
     if (j_first < nsteps) load_scales(rb, c, 0);
 
-    pdl_wait();  // x, Y and the workspace may belong to the previous kernel in the stream
+    if constexpr (!CHAIN) {
+        pdl_wait();  // x, Y and the workspace may belong to the previous kernel in the stream
+    } else if (op > 0) {
+        // every CTA must have delivered operation op - 1: `sync` counts arrivals since the kernel started
+        if (threadIdx.x == 0) {
+            const unsigned need = (unsigned)op * gridDim.x;
+            bool ok = false;
+            for (uint32_t i = 0; i < kSpinLimit && !ok; ++i) {
+                unsigned v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(sync) : "memory");
+                ok = v >= need;
+            }
+            if (!ok && err) atomicCAS(err, 0, 3 | (op << 8));
+        }
+        consumer_bar_sync<RG_CONSUMERS>();
+    }
     if constexpr (XSMEM) {
         uint4* dst = reinterpret_cast<uint4*>(smem + 1024);
         const uint4* src = reinterpret_cast<const uint4*>(X);
@@ -496,6 +543,43 @@ ring_kernel(const uint4* __restrict__ packed, const uint16_t* __restrict__ scale
         while (slot >= stages) { slot -= stages; phase ^= 1u; }
       }
     }
+    }  // consumers
+    if constexpr (CHAIN) {
+        __syncthreads();  // the CTA's part of this operation is delivered (and its ring and barriers are idle)
+        if (threadIdx.x == 0) {
+            __threadfence();
+            atomicAdd(sync, 1u);
+        }
+    }
+}
+
+template <int BITS, int MODE, int MT, int XMODE>
+__global__ void __launch_bounds__(rg_threads(MODE), 1)
+ring_kernel(const RingArgs ra, int* __restrict__ err) {
+    ring_body<BITS, MODE, MT, XMODE, false>(ra, err, nullptr, 0, 0);
+}
+
+// Persistent kernel over a list of dependent GEMVs (PoT codes, tiled layout, M = 1, activations staged in shared
+// memory): one launch instead of one per operation.  Launched cooperatively (all CTAs resident), since the CTAs wait
+// for one another between operations.  sync[0]: arrivals (see ring_body), sync[1]: CTAs that have finished the list;
+// the last of them puts both back to zero for the next launch.
+template <int BITS>
+__global__ void __launch_bounds__(rg_threads(RG_POT_MMA1), 1)
+ring_chain_kernel(const RingArgs* __restrict__ ops, int n_ops, unsigned* sync, int* __restrict__ err) {
+    int prev_stages = 0;
+    for (int op = 0; op < n_ops; ++op) {
+        const RingArgs ra = ops[op];
+        ring_body<BITS, RG_POT_MMA1, 1, 1, true>(ra, err, sync, op, prev_stages);
+        prev_stages = ra.stages;
+    }
+    if (threadIdx.x == 0) {
+        const unsigned d = atomicAdd(sync + 1, 1u);
+        if (d == gridDim.x - 1) {  // every CTA has left its last wait
+            sync[0] = 0u;
+            sync[1] = 0u;
+            __threadfence();
+        }
+    }
 }
 
 // Device error word shared by the ring kernels (0 = no bounded wait ever gave up).  One copy per
@@ -523,17 +607,28 @@ inline int ring_error_fetch() {
 }
 
 // Host side.  `err` may be nullptr.
+inline RingArgs ring_args(const RingPlan& p, const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
+                          int group, const void* X, int M, void* Y, void* workspace) {
+    RingArgs ra;
+    ra.packed = (const uint4*)packed;
+    ra.scales = (const uint16_t*)scales;
+    ra.zeros = (const uint16_t*)zeros;
+    ra.N = N; ra.K = K; ra.G = group; ra.spr = p.spr;
+    ra.total_steps = p.total_steps;
+    ra.stages = p.stages; ra.x_bytes = (int)p.x_bytes; ra.cmb_bytes = (int)p.cmb_bytes;
+    ra.X = (const __half*)X; ra.M = M; ra.Y = (__half*)Y;
+    ra.counters = (unsigned*)workspace;
+    ra.partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
+    return ra;
+}
 template <int BITS, int MODE, int MT>
 pot_status_t launch_ring(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                          const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
     const RingPlan p = plan_ring(N, K, M, BITS, MODE == RG_POT_MMA ? 8 * MT : 1, rg_groups(MODE));
     auto run = [&](auto kernel) -> pot_status_t {
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
-        unsigned* counters = (unsigned*)workspace;
-        float* partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
-        return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(rg_threads(MODE)), p.smem_bytes, s, (const uint4*)packed,
-                          (const uint16_t*)scales, (const uint16_t*)zeros, N, K, group, p.spr, p.total_steps, p.stages,
-                          (int)p.x_bytes, (int)p.cmb_bytes, (const __half*)X, M, (__half*)Y, partial, counters, err);
+        const RingArgs ra = ring_args(p, packed, scales, zeros, N, K, group, X, M, Y, workspace);
+        return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(rg_threads(MODE)), p.smem_bytes, s, ra, err);
     };
     if (p.x_in_smem) return run(ring_kernel<BITS, MODE, MT, 1>);
     return run(ring_kernel<BITS, MODE, MT, 0>);
