@@ -197,6 +197,40 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
                               int bits, int group, const void* x_f16, void* y_f16, void* stream);
 
 /*
+ * pot_gemv_chain_* -- a list of dependent pot_gemv operations (tiled layout, one `bits` for the
+ * whole list) executed by ONE persistent kernel instead of one launch per operation: between
+ * two decode GEMVs of a few microseconds, the end-of-grid / start-of-grid latency of separate
+ * launches costs as much as the arithmetic.  The kernel's CTAs stay resident, stream the next
+ * operation's weights while the current one finishes, and meet at a grid-wide arrival counter
+ * before they read the next activations, so operation i may read what operations < i wrote
+ * (y of one as x of the next).  The paper has no counterpart; the arithmetic and the result of
+ * every operation are those of pot_gemv (bit-identical).
+ *   - pot_gemv_chain_prepare checks every operation (as pot_gemv does), writes the list into
+ *     `scratch` (device memory, >= pot_gemv_chain_scratch_bytes(n_ops), 16-byte aligned) and zeroes
+ *     the kernel's counters there; call it once per list, outside of stream capture.  The ops
+ *     array is host memory and may be freed after the call returns.  POT_ERR_UNSUPPORTED when an
+ *     operation's K exceeds 32768 (its activations must fit the kernel's shared memory).
+ *   - pot_gemv_chain_run launches the kernel (cooperatively: all CTAs resident) on `stream`; it
+ *     may be called any number of times after one prepare, with the same n_ops and bits.  Each
+ *     operation's workspace must be zero before the first run (the kernel leaves it zero), and
+ *     two operations may share a workspace.  Runs of one scratch must not overlap.
+ */
+typedef struct {
+    const void* packed_tiled;   /* device, tiled layout                                   */
+    const void* scales_f16;     /* device [N, K/group]                                    */
+    int64_t N, K;
+    int group;
+    const void* x_f16;          /* device [K]                                             */
+    void* y_f16;                /* device [N]                                             */
+    void* workspace;            /* device, >= pot_gemv_workspace_bytes(N,K,bits,group)    */
+    size_t workspace_bytes;
+} pot_gemv_op_t;
+size_t pot_gemv_chain_scratch_bytes(int n_ops);
+pot_status_t pot_gemv_chain_prepare(const pot_gemv_op_t* ops_host, int n_ops, int bits, void* scratch,
+                                    size_t scratch_bytes, void* stream);
+pot_status_t pot_gemv_chain_run(const void* scratch, int n_ops, int bits, void* stream);
+
+/*
  * pot_gemm -- Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
  * accumulation, FP16 output.  M <= 8 (decode batches) runs a bandwidth-bound tensor-core
  * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the

@@ -1,3 +1,4 @@
+#include <vector>
 // Batch-1 decode GEMV, y = W~ x, fused with the dequantization (weights never touch HBM as
 // FP16).  CUDA-core kernels: codes are decoded in registers by the integer-add trick of
 // Sec. 4.2, products are accumulated in FP32 with the mixed-precision FMA
@@ -209,6 +210,74 @@ extern "C" pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* s
     const size_t counters_bytes = plan_ring(N, K, 1, bits, 1).ws_counters;
     if (cudaMemsetAsync(scratch, 0, counters_bytes, (cudaStream_t)stream) != cudaSuccess) return POT_ERR_CUDA;
     return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, need, stream);
+}
+
+// ---- chain of dependent GEMVs in one persistent kernel --------------------------------------------------
+constexpr size_t kChainHeader = 256;            // sync words of the kernel, then the operations
+constexpr size_t kChainSmem = 200 * 1024;       // every plan fits (plan_ring budgets 200 KB)
+
+extern "C" size_t pot_gemv_chain_scratch_bytes(int n_ops) {
+    return n_ops > 0 ? kChainHeader + (size_t)n_ops * sizeof(RingArgs) : 0;
+}
+
+extern "C" pot_status_t pot_gemv_chain_prepare(const pot_gemv_op_t* ops, int n_ops, int bits, void* scratch,
+                                               size_t scratch_bytes, void* stream) {
+    if (!ops || !scratch) return POT_ERR_NULL;
+    if (n_ops <= 0 || n_ops > (1 << 20)) return POT_ERR_SHAPE;
+    if (scratch_bytes < pot_gemv_chain_scratch_bytes(n_ops)) return POT_ERR_WORKSPACE;
+    if (!aligned16(scratch)) return POT_ERR_ALIGN;
+    std::vector<RingArgs> args((size_t)n_ops);
+    for (int i = 0; i < n_ops; ++i) {
+        const pot_gemv_op_t& o = ops[i];
+        if (!o.packed_tiled || !o.scales_f16 || !o.x_f16 || !o.y_f16) return POT_ERR_NULL;
+        const pot_status_t st = check_shape(o.N, o.K, bits, o.group);
+        if (st != POT_OK) return st;
+        if (o.N % 16 != 0) return POT_ERR_SHAPE;
+        if (!aligned16(o.packed_tiled) || !aligned16(o.scales_f16) || !aligned16(o.x_f16) || !aligned16(o.y_f16) ||
+            !aligned16(o.workspace))
+            return POT_ERR_ALIGN;
+        const RingPlan p = plan_ring(o.N, o.K, 1, bits, 1, rg_groups(RG_POT_MMA1));
+        if (!p.x_in_smem) return POT_ERR_UNSUPPORTED;
+        if (p.smem_bytes > kChainSmem) return POT_ERR_UNSUPPORTED;
+        if (p.ws_bytes > 0 && (!o.workspace || o.workspace_bytes < p.ws_bytes)) return POT_ERR_WORKSPACE;
+        args[(size_t)i] = ring_args(p, o.packed_tiled, o.scales_f16, nullptr, o.N, o.K, o.group, o.x_f16, 1, o.y_f16, o.workspace);
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, kChainHeader, s) != cudaSuccess) return POT_ERR_CUDA;
+    // pageable source: the runtime has consumed `args` when the call returns
+    if (cudaMemcpyAsync((char*)scratch + kChainHeader, args.data(), args.size() * sizeof(RingArgs), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+        return POT_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return POT_ERR_CUDA;
+    return POT_OK;
+}
+
+extern "C" pot_status_t pot_gemv_chain_run(const void* scratch, int n_ops, int bits, void* stream) {
+    if (!scratch) return POT_ERR_NULL;
+    if (n_ops <= 0) return POT_ERR_SHAPE;
+    if (bits < 2 || bits > 4) return POT_ERR_UNSUPPORTED;
+    unsigned* sync = (unsigned*)scratch;
+    const RingArgs* ops = (const RingArgs*)((const char*)scratch + kChainHeader);
+    int* err = ring_error_ptr();
+    auto run = [&](auto kernel) -> pot_status_t {
+        if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kSmCount);
+        cfg.blockDim = dim3(rg_threads(RG_POT_MMA1));
+        cfg.dynamicSmemBytes = kChainSmem;
+        cfg.stream = (cudaStream_t)stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;  // the CTAs wait for one another: all must be resident
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ops, n_ops, sync, err);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return e == cudaSuccess ? POT_OK : POT_ERR_CUDA;
+    };
+    if (bits == 2) return run(ring_chain_kernel<2>);
+    if (bits == 3) return run(ring_chain_kernel<3>);
+    return run(ring_chain_kernel<4>);
 }
 
 // Diagnostic: reads and clears the device error word of the gemv kernels in this library (0 = every bounded
