@@ -397,6 +397,28 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
     del g2, layers2
     torch.cuda.empty_cache()
 
+    # the headline chain through pot_gemv_chain: one persistent cooperative kernel per step instead of a graph of
+    # 160 programmatically chained launches
+    layersc, bytesc = build_chain(HEADLINE_BITS)
+    ops = [(t, sc, pr.K, GROUP, x, y, ws) for layer in layersc for (pr, t, sc, x, y, ws) in layer]
+    scratch = B.pot_gemv_chain_prepare(ops, HEADLINE_BITS, stream)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            B.pot_gemv_chain_run(scratch, len(ops), HEADLINE_BITS, stream)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(5, args.steps // 2)
+        e0.record(stream)
+        for _ in range(reps):
+            B.pot_gemv_chain_run(scratch, len(ops), HEADLINE_BITS, stream)
+        e1.record(stream)
+        stream.synchronize()
+    msc = e0.elapsed_time(e1) / reps
+    ex["chain_3bit_one_persistent_kernel"] = {"GBps": bytesc / msc / 1e6, "ms_per_step": msc,
+                                              "frac_of_measured_hbm": bytesc / msc / 1e6 / hbm, "launches_per_step": 1}
+    del scratch, ops, layersc
+    torch.cuda.empty_cache()
+
     # the same 3-bit chain with gate and up stored as one 4096 -> 22016 matrix (they share their input, as qkv do):
     # 128 launches per step instead of 160 over the same weights
     fused = (synth.LLAMA2_7B[0], synth.LLAMA2_7B[1], synth.Projection("gate_up", 4096, 22016), synth.LLAMA2_7B[4])
