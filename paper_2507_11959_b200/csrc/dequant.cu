@@ -78,6 +78,47 @@ __global__ void __launch_bounds__(DQ_THREADS) pot_dequant_kernel(const uint32_t*
     }
 }
 
+// PoT, n = 3: the 24-bit pieces of the canonical stream straddle 32-bit words, so the generic kernel needs two
+// loads per piece.  Here a thread takes four consecutive pieces = exactly three words (one coalesced 12-byte
+// read) and the block transposes the decoded pieces through shared memory, so that the stores stay coalesced.
+template <int EBIT>
+__global__ void __launch_bounds__(DQ_THREADS) pot_dequant3_kernel(const uint32_t* __restrict__ packed,
+                                                                  const uint16_t* __restrict__ scales, int64_t n_pieces,
+                                                                  int ppg_shift, uint4* __restrict__ out) {
+    constexpr uint32_t QM2 = (uint32_t)qmax_of(3) * 0x10001u, SM2 = 4u * 0x10001u;
+    __shared__ uint4 tile[4 * DQ_THREADS];
+    const int t = threadIdx.x;
+    const int64_t base = (int64_t)blockIdx.x * (4 * DQ_THREADS);  // first piece of the block
+    const int64_t c0 = base + 4 * t;                              // this thread's four pieces (one scale group)
+    if (c0 < n_pieces) {
+        const uint32_t* w = packed + (int64_t)blockIdx.x * (3 * DQ_THREADS) + 3 * t;
+        const uint32_t w0 = __ldg(w), w1 = __ldg(w + 1), w2 = __ldg(w + 2);
+        uint32_t s16 = __ldg(scales + (c0 >> ppg_shift));
+        if (EBIT == 7) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
+        const uint32_t sc2 = s16 * 0x10001u;
+        const uint32_t v[4] = {w0 & 0xFFFFFFu, __funnelshift_r(w0, w1, 24) & 0xFFFFFFu, __funnelshift_r(w1, w2, 16) & 0xFFFFFFu,
+                               w2 >> 8};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t pr[4], o[4];
+            spread_pairs<3>(v[j], pr);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t e = (pr[i] & QM2) * (1u << EBIT) + sc2;
+                o[i] = (pr[i] & SM2) * (1u << 13) + e;
+            }
+            tile[j * DQ_THREADS + ((t + 2 * j) & (DQ_THREADS - 1))] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int o = i * DQ_THREADS + t;  // piece of the block, written by consecutive threads
+        const int tt = o >> 2, j = o & 3;
+        if (base + o < n_pieces) out[base + o] = tile[j * DQ_THREADS + ((tt + 2 * j) & (DQ_THREADS - 1))];
+    }
+}
+
 // uniform twin, packed-half arithmetic: q -> FP16 by splicing it under the exponent of 1024,
 // (1024 + q) - (1024 + z) is exact, one HMUL2 by the scale rounds once.
 template <int BITS>
@@ -170,7 +211,14 @@ extern "C" pot_status_t pot_dequant(const void* packed, const void* scales, int6
 #define POT_DQ(B)                                                                                     \
     if (out_dtype == POT_F16) pot_dequant_kernel<B, 10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O); \
     else pot_dequant_kernel<B, 7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
-    if (bits == 2) { POT_DQ(2) } else if (bits == 3) { POT_DQ(3) } else { POT_DQ(4) }
+    if (bits == 2) {
+        POT_DQ(2)
+    } else if (bits == 3) {
+        if (out_dtype == POT_F16) pot_dequant3_kernel<10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
+        else pot_dequant3_kernel<7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
+    } else {
+        POT_DQ(4)
+    }
 #undef POT_DQ
     return launched();
 }
