@@ -162,6 +162,45 @@ __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_fast_kernel(const uin
     }
 }
 
+// uniform twin, n = 3, same access pattern as pot_dequant3_kernel (three aligned words per thread, transposition
+// through shared memory): only the arithmetic differs
+__global__ void __launch_bounds__(DQ_THREADS) uint_dequant3_fast_kernel(const uint32_t* __restrict__ packed,
+                                                                        const uint16_t* __restrict__ scales,
+                                                                        const uint16_t* __restrict__ zeros, int64_t n_pieces,
+                                                                        int ppg_shift, uint4* __restrict__ out) {
+    __shared__ uint4 tile[4 * DQ_THREADS];
+    const int t = threadIdx.x;
+    const int64_t base = (int64_t)blockIdx.x * (4 * DQ_THREADS);
+    const int64_t c0 = base + 4 * t;
+    if (c0 < n_pieces) {
+        const uint32_t* w = packed + (int64_t)blockIdx.x * (3 * DQ_THREADS) + 3 * t;
+        const uint32_t w0 = __ldg(w), w1 = __ldg(w + 1), w2 = __ldg(w + 2);
+        const __half2 s2 = __half2half2(__ushort_as_half(__ldg(scales + (c0 >> ppg_shift))));
+        const __half2 zm2 = __hadd2(__half2half2(__ushort_as_half(__ldg(zeros + (c0 >> ppg_shift)))), __float2half2_rn(1024.0f));
+        const uint32_t v[4] = {w0 & 0xFFFFFFu, __funnelshift_r(w0, w1, 24) & 0xFFFFFFu, __funnelshift_r(w1, w2, 16) & 0xFFFFFFu,
+                               w2 >> 8};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t pr[4], o[4];
+            spread_pairs<3>(v[j], pr);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t h = pr[i] | 0x64006400u;  // half2{1024 + q0, 1024 + q1}
+                const __half2 wv = __hmul2(__hsub2(*reinterpret_cast<const __half2*>(&h), zm2), s2);
+                o[i] = *reinterpret_cast<const uint32_t*>(&wv);
+            }
+            tile[j * DQ_THREADS + ((t + 2 * j) & (DQ_THREADS - 1))] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int o = i * DQ_THREADS + t;
+        const int tt = o >> 2, j = o & 3;
+        if (base + o < n_pieces) out[base + o] = tile[j * DQ_THREADS + ((tt + 2 * j) & (DQ_THREADS - 1))];
+    }
+}
+
 // uniform twin, the textbook form: integer -> float, subtract the zero-point, multiply by the scale.
 template <int BITS>
 __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_naive_kernel(const uint32_t* __restrict__ packed,
@@ -241,7 +280,14 @@ extern "C" pot_status_t uint_dequant(const void* packed, const void* scales, con
 #define UINT_DQ(B)                                                                                              \
     if (kernel == UINT_KERNEL_FAST) uint_dequant_fast_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O); \
     else uint_dequant_naive_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
-    if (bits == 2) { UINT_DQ(2) } else if (bits == 3) { UINT_DQ(3) } else { UINT_DQ(4) }
+    if (bits == 2) {
+        UINT_DQ(2)
+    } else if (bits == 3) {
+        if (kernel == UINT_KERNEL_FAST) uint_dequant3_fast_kernel<<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
+        else uint_dequant_naive_kernel<3><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
+    } else {
+        UINT_DQ(4)
+    }
 #undef UINT_DQ
     return launched();
 }
