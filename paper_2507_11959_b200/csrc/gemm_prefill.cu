@@ -49,6 +49,9 @@ __device__ __forceinline__ uint64_t pf_smem_desc(uint32_t saddr) {
            ((uint64_t)2 << 61);
 }
 
+// the descriptor's high word does not depend on the address
+constexpr uint64_t PF_DESC_CONST = ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+
 __device__ __forceinline__ void pf_tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
                  "l"(map), "r"(x), "r"(y), "r"(bar)
@@ -60,6 +63,17 @@ __device__ __forceinline__ void pf_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// same, the two descriptors given as their low words + the common high word
+__device__ __forceinline__ void pf_mma2(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void pf_commit(uint32_t bar) {
@@ -119,6 +133,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         cb1 = ((int64_t)zsplit + 1) * (K / 128) / splits;
     }
     const int64_t ncb = K / 128;
+    // a tile with at most 128 real tokens (decode batches, the ragged last token tile) uses one accumulator only
+    const int n_mt = M - m0 > PF_BM ? PF_MT : 1;
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
@@ -149,36 +165,51 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
                 }
-                mbar_expect_tx(full(s), PF_MT * PF_ATOM_BYTES);
+                mbar_expect_tx(full(s), (uint32_t)n_mt * PF_ATOM_BYTES);
                 const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
 #pragma unroll
                 for (int mt = 0; mt < PF_MT; ++mt)
-                    pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
+                    if (mt < n_mt) pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------
         if (lane == 0) {
-            // A barrier test costs a few hundred cycles even when the phase is long complete, so the test for
-            // stage kb+1 is put in flight before the MMAs of stage kb are issued and only examined afterwards.
+            // One thread's dependent instructions retire every ~5 cycles, so everything the loop needs per MMA is
+            // prepared here: the low descriptor word of every stage's tiles (the high word is a constant) and the
+            // barrier addresses; the loop is unrolled over the stages so that these stay in registers and a K step
+            // is one add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the
+            // test for stage kb+1 is put in flight before the MMAs of stage kb are issued and examined afterwards.
+            uint32_t alo[PF_STAGES], blo[PF_STAGES];
+#pragma unroll
+            for (int s = 0; s < PF_STAGES; ++s) {
+                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
+                alo[s] = (uint32_t)pf_smem_desc(a);
+                blo[s] = (uint32_t)pf_smem_desc(a + PF_MT * PF_ATOM_BYTES);
+            }
+            constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
             uint32_t ready = mbar_test(full(0), 0);
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % PF_STAGES;
-                const uint32_t ph = (uint32_t)((kb / PF_STAGES) & 1);
-                if (!ready && !mbar_wait(full(s), ph)) {
-                    if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+            uint32_t ph = 0;
+            for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
+#pragma unroll
+                for (int s = 0; s < PF_STAGES; ++s) {
+                    const int kb = kb0 + s;
+                    if (kb >= nkb) break;
+                    if (!ready && !mbar_wait(full(s), ph)) {
+                        if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+                    }
+                    ready = 0;
+                    if (kb + 1 < nkb) ready = mbar_test(full((s + 1) % PF_STAGES), s + 1 == PF_STAGES ? ph ^ 1u : ph);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                    for (int mt = 0; mt < PF_MT; ++mt)
+#pragma unroll
+                        for (int ks = 0; ks < PF_BK / 16; ++ks)
+                            if (mt < n_mt)
+                                pf_mma2(tmem_base + (uint32_t)(mt * PF_BN), alo[s] + (uint32_t)((mt * PF_ATOM_BYTES + ks * 32) >> 4),
+                                        blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, PF_IDESC, (s | ks) != 0 ? 1u : (uint32_t)(kb0 != 0));
+                    pf_commit(empty(s));  // the stage is free again once these MMAs have read it
                 }
-                ready = 0;
-                if (kb + 1 < nkb) ready = mbar_test(full((kb + 1) % PF_STAGES), (uint32_t)(((kb + 1) / PF_STAGES) & 1));
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES), b = a + PF_MT * PF_ATOM_BYTES;
-#pragma unroll
-                for (int mt = 0; mt < PF_MT; ++mt)
-#pragma unroll
-                    for (int ks = 0; ks < PF_BK / 16; ++ks)
-                        pf_mma(tmem_base + (uint32_t)(mt * PF_BN), pf_smem_desc(a + mt * PF_ATOM_BYTES + ks * 32),
-                               pf_smem_desc(b + ks * 32), PF_IDESC, (kb | ks) != 0 ? 1u : 0u);
-                pf_commit(empty(s));  // the stage is free again once these MMAs have read it
             }
             pf_commit(accum);          // the accumulators are complete once every MMA has finished
         }
