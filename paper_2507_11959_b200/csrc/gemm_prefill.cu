@@ -1,26 +1,30 @@
 // Prefill GEMM on 5th-generation tensor cores: Y[M,N] = X[M,K] W~^T, FP16 in, FP32 accumulate in
 // tensor memory, FP16 out, with the PoT dequantization fused in (tiled weight layout).
 //
-// One CTA computes a 256-token x 128-feature tile of Y as two 128 x 128 accumulators that share every
-// decoded weight tile.  Per 64-wide K block (one pipeline stage, 48 KB):
+// One CTA (one per SM) computes a 256-token x 128-feature tile of Y.  Per 64-wide K block (one pipeline stage, 48 KB;
+// four stages):
 //   warp 0 (one lane)  : TMA loads of the two X tiles (64-column boxes, 128-byte swizzle) into the stage;
-//   warps 2..9         : "dequant producers" -- each thread fetches the 32 codes of one weight row that the
-//                        stage needs (16-byte loads from the tiled layout), decodes them in registers
-//                        with the mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the
-//                        stage's B tile in exactly the layout the tensor core expects (K-major, 8-row x
-//                        128-byte atoms, 16-byte chunks XOR-swizzled with the row index), then
-//                        fence.proxy.async + mbarrier arrive;
-//   warp 1 (one lane)  : waits for both operands, issues 2 x 4 tcgen05.mma (M = 128, N = 128, K = 16) whose
-//                        accumulators live in 2 x 128 columns of tensor memory, and tcgen05.commit's the
-//                        stage back to the producers.
-// After the last K block the accumulators are committed to a barrier; warps 2..9 read them with
-// tcgen05.ld (each warp its own 32-lane quarter of one accumulator), convert to FP16 and store.  The
-// weights are re-decoded once per 256-token tile (M / 256 times overall), which is the price of never
-// writing FP16 weights to HBM.
+//   warps 4..19        : "dequant producers", four groups of four warps that take the stages in turn -- each thread
+//                        fetches the 32 codes of one weight row that the stage needs (8-byte loads from the tiled
+//                        layout, prefetched three of the group's stages ahead), decodes them in registers with the
+//                        mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the stage's B tile in
+//                        exactly the layout the tensor core expects (K-major, 8-row x 128-byte atoms, 16-byte chunks
+//                        XOR-swizzled with the row index), then fence.proxy.async + mbarrier arrive;
+//   warps 1, 2 (one lane each) : the two MMA issuers take alternate stages; each waits for both operands, issues
+//                        2 x 4 tcgen05.mma (M = 128, N = 128, K = 16) into ITS OWN pair of 128-column accumulators
+//                        in tensor memory and tcgen05.commit's the stage back to the producers.  One issuing thread
+//                        leaves the tensor pipe idle for several hundred cycles per stage (barrier test, fence,
+//                        commit, the pipe's start-up after a gap); two threads fill each other's gaps.
+// After the last K block each issuer commits to a common barrier; the producer warps read the accumulators with
+// tcgen05.ld (each warp its own 32-lane quarter), add the two issuers' sums in a fixed order, convert to FP16 and
+// store.  The weights are re-decoded once per 256-token tile (M / 256 times overall), which is the price of never
+// writing FP16 weights to HBM.  A tile with at most 128 real tokens uses one accumulator per issuer only.
 //
 // All mbarrier waits are bounded (see ring.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "layout.cuh"
@@ -32,8 +36,10 @@ constexpr int PF_BM = 128;      // tokens per accumulator (MMA M)
 constexpr int PF_MT = 2;        // accumulators per CTA: 256 tokens share one decoded weight tile
 constexpr int PF_BN = 128;      // features per tile (MMA N)
 constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte swizzle atom wide)
-constexpr int PF_PRODUCERS = 8;                      // dequant / epilogue warps
-constexpr int PF_THREADS = (2 + PF_PRODUCERS) * 32;  // + TMA warp + MMA warp
+// Warps: 0 = TMA, 1 .. NI = MMA issuers, then (from a warp index that is a multiple of 2 or 4, so that warp & 3 walks the
+// tensor-memory lane quarters in step) NG groups of four dequant / epilogue warps.
+__host__ __device__ constexpr int pf_prod_warp0(int ni) { return ni == 2 ? 4 : 2; }
+__host__ __device__ constexpr int pf_threads(int ng, int ni) { return (pf_prod_warp0(ni) + 4 * ng) * 32; }
 constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
 constexpr int PF_STAGE_BYTES = (PF_MT + 1) * PF_ATOM_BYTES;  // two X tiles + one weight tile
 constexpr size_t pf_smem_bytes(int stages) { return 1024 /*align slack*/ + (size_t)stages * PF_STAGE_BYTES + 256 /*barriers*/; }
@@ -76,6 +82,18 @@ __device__ __forceinline__ void pf_mma2(uint32_t d_tmem, uint32_t alo, uint32_t 
         "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The producers' prefetch loads as volatile statements: issued exactly once and where the source puts them (ahead of the
+// wait for the stage), never re-materialised behind it.
+__device__ __forceinline__ uint2 pf_ldg_v2(const uint2* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t pf_ldg_u16(const uint16_t* p) {
+    uint16_t v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return (uint32_t)v;
+}
 __device__ __forceinline__ void pf_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -91,10 +109,56 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "memory");
 }
 
-// PF_STAGES = 2: two CTAs share an SM and hide each other's hand-off latencies (large M, many tiles);
-// PF_STAGES = 4: one CTA per SM with a deeper pipeline (few tiles, e.g. decode batches of 9..256 tokens).
-template <int BITS, int PF_STAGES>
-__global__ void __launch_bounds__(PF_THREADS, PF_STAGES == 2 ? 2 : 1)
+// The MMA issuer J of NI (one thread): takes the stages kb = J, J + NI, ... of the CTA's nkb stages and accumulates them
+// into its own pair of accumulators.  One thread's dependent instructions retire every ~5 cycles and the tensor pipe
+// idles meanwhile, so what the loop needs per MMA is prepared first: the low descriptor word of every stage's tiles (the
+// high word is a constant); the loop is unrolled over the stages so that these stay in registers and a K step is one
+// add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the test for the issuer's
+// next stage is put in flight before the MMAs of this one are issued and examined afterwards.
+template <int J, int NI, int PF_STAGES>
+__device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, int n_mt, int* err) {
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
+    const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
+    uint32_t alo[PF_STAGES], blo[PF_STAGES];
+#pragma unroll
+    for (int s = 0; s < PF_STAGES; ++s) {
+        const uint32_t a = smem0 + (uint32_t)s * PF_STAGE_BYTES;
+        alo[s] = (uint32_t)pf_smem_desc(a);
+        blo[s] = (uint32_t)pf_smem_desc(a + PF_MT * PF_ATOM_BYTES);
+    }
+    constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
+    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BN * PF_MT);
+    uint32_t ready = mbar_test(full(J), 0);
+    uint32_t ph = 0;
+    for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
+#pragma unroll
+        for (int s = J; s < PF_STAGES; s += NI) {
+            const int kb = kb0 + s;
+            if (kb >= nkb) break;
+            if (!ready && !mbar_wait(full(s), ph)) {
+                if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+            }
+            ready = 0;
+            if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int mt = 0; mt < PF_MT; ++mt)
+#pragma unroll
+                for (int ks = 0; ks < PF_BK / 16; ++ks)
+                    if (mt < n_mt)
+                        pf_mma2(d0 + (uint32_t)(mt * PF_BN), alo[s] + (uint32_t)((mt * PF_ATOM_BYTES + ks * 32) >> 4),
+                                blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, PF_IDESC, (s != J || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
+            pf_commit(empty(s));  // the stage is free again once these MMAs have read it
+        }
+    }
+    pf_commit(accum);  // this issuer's accumulators are complete once all its MMAs have finished
+}
+
+// PF_STAGES stages, NG producer groups (a stage buffer always belongs to the same group), NI issuers with their own
+// accumulators.  Instantiated as <bits, 4, 4, 2>.
+template <int BITS, int PF_STAGES, int NG, int NI>
+__global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
                         __half* __restrict__ Y, float* __restrict__ partial, unsigned* __restrict__ counters,
@@ -110,6 +174,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
     const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
 
+    constexpr int PROD_WARP0 = pf_prod_warp0(NI);
+    constexpr int NPT = NG * 128;                       // producer / epilogue threads
+    constexpr int TMEM_COLS = NI * PF_BN * PF_MT;       // one pair of accumulators per issuer
+    static_assert(PF_STAGES % NG == 0 && NG % 2 == 0 && PF_STAGES % NI == 0, "a stage buffer belongs to one group and one issuer");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
     // into tail_splits items along K, so that the last, partly filled wave of CTAs is short.  Tiles are numbered
@@ -140,14 +208,14 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
-            mbar_init(full(s), 1 + PF_PRODUCERS / 2);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
+            mbar_init(full(s), 1 + 4);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
             mbar_init(empty(s), 1);
         }
-        mbar_init(accum, 1);
+        mbar_init(accum, NI);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {  // allocate 256 columns of tensor memory (whole warp), base address lands in shared memory
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(PF_BN * PF_MT) : "memory");
+    if (warp == 1) {  // allocate the accumulator columns of tensor memory (whole warp), base address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -172,55 +240,20 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     if (mt < n_mt) pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ---------------------------------------------------------------
+    } else if (warp <= NI) {
+        // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            // One thread's dependent instructions retire every ~5 cycles, so everything the loop needs per MMA is
-            // prepared here: the low descriptor word of every stage's tiles (the high word is a constant) and the
-            // barrier addresses; the loop is unrolled over the stages so that these stay in registers and a K step
-            // is one add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the
-            // test for stage kb+1 is put in flight before the MMAs of stage kb are issued and examined afterwards.
-            uint32_t alo[PF_STAGES], blo[PF_STAGES];
-#pragma unroll
-            for (int s = 0; s < PF_STAGES; ++s) {
-                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
-                alo[s] = (uint32_t)pf_smem_desc(a);
-                blo[s] = (uint32_t)pf_smem_desc(a + PF_MT * PF_ATOM_BYTES);
-            }
-            constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
-            uint32_t ready = mbar_test(full(0), 0);
-            uint32_t ph = 0;
-            for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
-#pragma unroll
-                for (int s = 0; s < PF_STAGES; ++s) {
-                    const int kb = kb0 + s;
-                    if (kb >= nkb) break;
-                    if (!ready && !mbar_wait(full(s), ph)) {
-                        if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
-                    }
-                    ready = 0;
-                    if (kb + 1 < nkb) ready = mbar_test(full((s + 1) % PF_STAGES), s + 1 == PF_STAGES ? ph ^ 1u : ph);
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-                    for (int mt = 0; mt < PF_MT; ++mt)
-#pragma unroll
-                        for (int ks = 0; ks < PF_BK / 16; ++ks)
-                            if (mt < n_mt)
-                                pf_mma2(tmem_base + (uint32_t)(mt * PF_BN), alo[s] + (uint32_t)((mt * PF_ATOM_BYTES + ks * 32) >> 4),
-                                        blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, PF_IDESC, (s | ks) != 0 ? 1u : (uint32_t)(kb0 != 0));
-                    pf_commit(empty(s));  // the stage is free again once these MMAs have read it
-                }
-            }
-            pf_commit(accum);          // the accumulators are complete once every MMA has finished
+            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
+            else pf_issue<NI - 1, NI, PF_STAGES>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
         }
-    } else {
+    } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
-        // Two groups of four warps take alternate stages: a stage visit costs a warp a fixed ~1000 cycles of
+        // NG groups of four warps take the stages in turn: a stage visit costs a warp a fixed ~1000 cycles of
         // hand-off latency (barrier test, proxy fence, arrive), so more stages must be in preparation at once.
         // Stage kb covers columns 64*kb .. 64*kb+63, i.e. half (kb & 1) of column block kb / 2; group g owns the
-        // stages with kb & 1 == g, hence always the same half of the records.  Thread = one weight row.
-        const int pt = threadIdx.x - 64;          // 0..255
-        const int grp = pt >> 7, row = pt & 127;
+        // stages with kb % NG == g, hence (NG is even) always the same half of the records.  Thread = one weight row.
+        const int pt = threadIdx.x - 32 * PROD_WARP0;          // 0 .. NPT-1
+        const int grp = pt >> 7, row = pt & 127, half = grp & 1;
         const int64_t n = n0 + row;
         const bool row_ok = n < N;
         const int64_t rb = n >> 4;
@@ -228,7 +261,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         const int gpr = (int)(K / G), spg = 128 / G;
         // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.  Every 16-byte plane of the
         // row holds one word of each quarter; the group needs quarters 2*grp and 2*grp + 1: 8 bytes per plane.
-        constexpr int PF_DEPTH = (BITS == 4 && PF_STAGES == 2) ? 3 : 4;  // 4-bit records at 96 registers: one buffer fewer
+        constexpr int PF_DEPTH = 4;
         uint32_t rec[PF_DEPTH][2 * BITS];
         uint32_t sc2[PF_DEPTH];
         auto load = [&](int kb, int buf) {
@@ -236,28 +269,31 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cb0 + (kb >> 1)) * (16 * BITS));
 #pragma unroll
                 for (int t = 0; t < BITS; ++t) {
-                    const uint2 q = __ldg(unit + (t * 16 + r) * 2 + grp);
+                    const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
                     rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
                 }
-                const int64_t so = n * gpr + (cb0 + (kb >> 1)) * spg + (spg == 2 ? grp : 0);
-                sc2[buf] = (uint32_t)__ldg(scales + so);  // raw bits: any arithmetic here would stall on the load
+                const int64_t so = n * gpr + (cb0 + (kb >> 1)) * spg + (spg == 2 ? half : 0);
+                sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
-        const int nmine = (nkb - grp + 1) / 2;   // stages kb = grp, grp + 2, ...
+        const int nmine = nkb > grp ? (nkb - grp + NG - 1) / NG : 0;   // stages kb = grp, grp + NG, ...
 #pragma unroll
         for (int p = 0; p < PF_DEPTH - 1; ++p)
-            if (p < nmine) load(2 * p + grp, p);
+            if (p < nmine) load(NG * p + grp, p);
         for (int i4 = 0; i4 < nmine; i4 += PF_DEPTH) {
 #pragma unroll
             for (int buf = 0; buf < PF_DEPTH; ++buf) {
                 const int i = i4 + buf;
                 if (i >= nmine) break;
-                const int kb = 2 * i + grp;
-                if (i + PF_DEPTH - 1 < nmine) load(kb + 2 * (PF_DEPTH - 1), (buf + PF_DEPTH - 1) % PF_DEPTH);
+                const int kb = NG * i + grp;
+                if (i + PF_DEPTH - 1 < nmine) load(kb + NG * (PF_DEPTH - 1), (buf + PF_DEPTH - 1) % PF_DEPTH);
                 const int s = kb % PF_STAGES;
-                if (kb >= PF_STAGES) {  // one lane polls for the whole warp: the warp is about to WRITE the stage
-                    if (lane == 0 && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
-                        if (err) atomicCAS(err, 0, 0x30 | (kb << 8));
+                if (kb >= PF_STAGES) {
+                    // Every lane polls (the warp is about to WRITE the stage).  One polling lane + __syncwarp() left the
+                    // warp running as two groups (lane 0 / the rest) through the whole decode in some builds: every
+                    // load and store issued twice.
+                    if (!mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
+                        if (err && lane == 0) atomicCAS(err, 0, 0x30 | (kb << 8));
                     }
                     __syncwarp();
                 }
@@ -290,7 +326,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
-        const int mt = (warp - 2) >> 2;           // warps 2..5 read accumulator 0, warps 6..9 accumulator 1
+        const int ew = warp - PROD_WARP0;
+        const int mt = (ew >> 2) & 1;             // four warps per accumulator; with NG = 4 two sets of them share the columns
+        constexpr int CHUNKS = (PF_BN / 32) / (NG / 2);
+        const int cc0 = (ew >> 3) * CHUNKS;
         const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
         int tile, zsplit, splits;  // recomputed here rather than kept in registers across the main loop
         item(tile, zsplit, splits);
@@ -315,11 +354,20 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             }
         };
 #pragma unroll
-        for (int cc = 0; cc < PF_BN / 32; ++cc) {
-            const int col = cc * 32;
+        for (int cc = 0; cc < CHUNKS; ++cc) {
+            if (mt >= n_mt) break;                // (warp-uniform) no token of this accumulator exists
+            const int col = (cc0 + cc) * 32;
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(mt * PF_BN + col), v);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (NI == 2) {                        // add the second issuer's sums (odd stages) to the first's: a fixed order
+                uint32_t v1[32];
+                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BN * PF_MT + mt * PF_BN + col), v1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
+            } else {
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            }
             if (token < M) {
                 if (splits == 1) {
                     store_row(v, col);
@@ -336,25 +384,24 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             // ascending order -- the result does not depend on timing -- and writes Y.
             __shared__ unsigned s_prev;
             __threadfence();
-            asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
-            if (threadIdx.x == 64) s_prev = atomicAdd(&counters[tail_index], 1u);
-            asm volatile("bar.sync 2, %0;" ::"n"(PF_PRODUCERS * 32) : "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(NPT) : "memory");
+            if (threadIdx.x == 32 * PROD_WARP0) s_prev = atomicAdd(&counters[tail_index], 1u);
+            asm volatile("bar.sync 2, %0;" ::"n"(NPT) : "memory");
             if (s_prev == (unsigned)splits - 1u) {
                 __threadfence();
-                // The 256 epilogue threads walk the tile in 16-byte pieces, consecutive threads on consecutive
+                // The epilogue threads walk the tile in 16-byte pieces, consecutive threads on consecutive
                 // pieces (coalesced), four pieces per thread in flight; the splits are added in ascending order.
-                const int pt = threadIdx.x - 64;
                 const float* tile0 = partial + (int64_t)tail_index * splits * rows_alloc * PF_BN;
                 const int64_t split_stride = rows_alloc * PF_BN;
                 const int npieces = (int)(rows_alloc * PF_BN / 4);
-                for (int p0 = pt; p0 < npieces; p0 += 4 * PF_PRODUCERS * 32) {
+                for (int p0 = pt; p0 < npieces; p0 += 4 * NPT) {
                     float4 acc4[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) acc4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int z = 0; z < splits; ++z) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            const int pc = p0 + u * PF_PRODUCERS * 32;
+                            const int pc = p0 + u * NPT;
                             if (pc < npieces) {
                                 const float4 t = __ldcg(reinterpret_cast<const float4*>(tile0 + z * split_stride) + pc);
                                 acc4[u].x += t.x; acc4[u].y += t.y; acc4[u].z += t.z; acc4[u].w += t.w;
@@ -363,7 +410,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const int pc = p0 + u * PF_PRODUCERS * 32;
+                        const int pc = p0 + u * NPT;
                         const int64_t row = m0 + pc / (PF_BN / 4), colx = n0 + 4 * (pc % (PF_BN / 4));
                         if (pc < npieces && row < M && colx < N) {  // N % 16 == 0: a piece is inside or outside as a whole
                             const __half2 h0 = __floats2half2_rn(acc4[u].x, acc4[u].y), h1 = __floats2half2_rn(acc4[u].z, acc4[u].w);
@@ -372,7 +419,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                         }
                     }
                 }
-                if (threadIdx.x == 64) counters[tail_index] = 0u;  // leave the workspace ready for the next call
+                if (threadIdx.x == 32 * PROD_WARP0) counters[tail_index] = 0u;  // leave the workspace ready for the next call
             }
         }
     }
@@ -381,7 +428,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(PF_BN * PF_MT) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(TMEM_COLS) : "memory");
     }
 }
 
@@ -407,9 +454,9 @@ bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group
     // TMA needs the X row pitch (2K bytes) to be a multiple of 16 -- implied by K % 128 == 0 -- and 32-bit box coordinates
     return M > 0 && N % 16 == 0 && K % 128 == 0 && M < (int64_t(1) << 31) && K < (int64_t(1) << 31);
 }
-// How the output tiles become work items.  Tiles run two CTAs per SM (296 slots); the tiles of the last, partly
-// filled wave -- or all tiles when they cover less than half of the SMs -- are cut along K into `splits` items
-// each (FP32 partial sums + an arrival counter per such tile in the workspace), at least four column blocks per item.
+// How the output tiles become work items.  One CTA per SM (148 slots); the tiles of the last, partly filled wave -- or all
+// tiles when they cover at most half of the SMs -- are cut along K into `splits` items each (FP32 partial sums + an
+// arrival counter per such tile in the workspace), at least four column blocks per item.
 struct PrefillPlan {
     int tiles_m, tiles, n_full, n_tail, splits;
     int64_t rows_alloc;
@@ -419,10 +466,10 @@ static PrefillPlan prefill_plan(int64_t M, int64_t N, int64_t K) {
     PrefillPlan p{};
     p.tiles_m = (int)((M + PF_BM * PF_MT - 1) / (PF_BM * PF_MT));
     p.tiles = p.tiles_m * (int)((N + PF_BN - 1) / PF_BN);
-    const int slots = 2 * kSmCount;
+    const int slots = kSmCount;
     const int rem = p.tiles % slots;
     int tail = 0;
-    if (2 * p.tiles <= kSmCount) tail = p.tiles;            // small problem: every tile is split
+    if (2 * p.tiles <= slots) tail = p.tiles;            // small problem: every tile is split
     else if (p.tiles > slots && rem > 0 && 2 * rem <= slots) tail = rem;  // the last wave fills at most half of the slots
     int64_t s = tail > 0 ? slots / tail : 1;
     const int64_t max_by_k = (K / 128) / 4;
@@ -460,23 +507,18 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
-    const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits)), block(PF_THREADS);
-    // too few CTAs to fill two per SM: one CTA per SM with the deeper pipeline
-    const bool deep = (int64_t)grid.x <= 2 * kSmCount && pl.n_tail == 0;
-    auto run = [&](auto kernel, int stages) -> pot_status_t {
-        const size_t smem = pf_smem_bytes(stages);
+    const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits));
+    auto run = [&](auto kernel) -> pot_status_t {
+        const size_t smem = pf_smem_bytes(4);
+        const dim3 block((unsigned)pf_threads(4, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (__half*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
-    if (deep) {
-        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4>, 4);
-        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4>, 4);
-        return run(pot_gemm_prefill_kernel<4, 4>, 4);
-    }
-    if (bits == 2) return run(pot_gemm_prefill_kernel<2, 2>, 2);
-    if (bits == 3) return run(pot_gemm_prefill_kernel<3, 2>, 2);
-    return run(pot_gemm_prefill_kernel<4, 2>, 2);
+    // four stages, four producer groups, two issuers: one CTA per SM
+    if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2>);
+    if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2>);
+    return run(pot_gemm_prefill_kernel<4, 4, 4, 2>);
 }
 
 static int* prefill_error_ptr() { return ring_error_ptr(); }

@@ -47,11 +47,12 @@ def test_size_helpers(L):
     assert ws == 1024 + 256 * 22 * 16 * 4 and ws % 16 == 0
     assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
     # M > 8 runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
-    # cover less than half of the SMs (32 tiles -> 9 splits of 32 token rows x 128 features), or those of a last
-    # wave that fills at most half of the 296 CTA slots (640 tiles -> 48 tail tiles x 6 splits x 256 rows).
-    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 32 * 9 * 32 * 128 * 4
-    assert L.pot_gemm_workspace_bytes(2048, 10240, 8192, 3, 128) == 256 + 48 * 6 * 256 * 128 * 4
-    assert L.pot_gemm_workspace_bytes(2048, 8192, 28672, 3, 128) == 0     # 512 tiles: the last wave is 73 % full
+    # cover at most half of the SMs (32 tiles -> 4 splits of 32 token rows x 128 features), or those of a last
+    # wave that fills at most half of the 148 CTA slots (640 tiles -> 48 tail tiles x 3 splits x 256 rows).
+    assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 32 * 4 * 32 * 128 * 4
+    assert L.pot_gemm_workspace_bytes(2048, 10240, 8192, 3, 128) == 256 + 48 * 3 * 256 * 128 * 4
+    assert L.pot_gemm_workspace_bytes(2048, 8192, 28672, 3, 128) == 512 + 68 * 2 * 256 * 128 * 4  # 512 tiles: 68 in the last wave
+    assert L.pot_gemm_workspace_bytes(2048, 3584, 8192, 3, 128) == 0     # 224 tiles: the last wave is 51 % full
 
 
 def test_status_strings(L):
