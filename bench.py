@@ -526,9 +526,16 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
             g = capture(lambda s: B.pot_gemm(P, S, pr.K, bits, GROUP, X, layout, Y=Y, workspace=ws, stream=s))
             t = min(time_graph(g, 3, 3) for _ in range(2))
             fl = 2.0 * synth.PREFILL_M * pr.N * pr.K
-            rows.append({"shape": f"70B {pr.name} {pr.K}->{pr.N}", "M": synth.PREFILL_M, "bits": bits, "ms": t,
-                         "TFLOPs": fl / t / 1e9, "frac_tensor_sustained": fl / t / 1e9 / peaks["bf16_tflops_sustained"],
-                         "kernel": "tcgen05" if layout == B.TILED else "mma.sync fallback"})
+            row = {"shape": f"70B {pr.name} {pr.K}->{pr.N}", "M": synth.PREFILL_M, "bits": bits, "ms": t,
+                   "TFLOPs": fl / t / 1e9, "frac_tensor_burst": fl / t / 1e9 / peaks["bf16_tflops"],
+                   "kernel": "tcgen05" if layout == B.TILED else "mma.sync fallback"}
+            if bits == HEADLINE_BITS and pr.name == "gate_or_up":
+                # the same launch ~600 times back to back: about half a second under the power cap, the regime in
+                # which the sustained cuBLAS figure was measured
+                ts = time_graph(g, 600, 3)
+                row.update({"ms_sustained": ts, "TFLOPs_sustained": fl / ts / 1e9,
+                            "frac_tensor_sustained": fl / ts / 1e9 / peaks["bf16_tflops_sustained"]})
+            rows.append(row)
             del g
         del W, X, Y
         torch.cuda.empty_cache()

@@ -41,8 +41,9 @@ constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte s
 __host__ __device__ constexpr int pf_prod_warp0(int ni) { return ni == 2 ? 4 : 2; }
 __host__ __device__ constexpr int pf_threads(int ng, int ni) { return (pf_prod_warp0(ni) + 4 * ng) * 32; }
 constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
-constexpr int PF_STAGE_BYTES = (PF_MT + 1) * PF_ATOM_BYTES;  // two X tiles + one weight tile
-constexpr size_t pf_smem_bytes(int stages) { return 1024 /*align slack*/ + (size_t)stages * PF_STAGE_BYTES + 256 /*barriers*/; }
+// a stage: MT X tiles (token tiles) + one weight tile
+__host__ __device__ constexpr int pf_stage_bytes(int mt) { return (mt + 1) * PF_ATOM_BYTES; }
+constexpr size_t pf_smem_bytes(int stages, int mt) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt) + 256 /*barriers*/; }
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
 constexpr uint32_t PF_IDESC = (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ |
@@ -115,7 +116,7 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // high word is a constant); the loop is unrolled over the stages so that these stay in registers and a K step is one
 // add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the test for the issuer's
 // next stage is put in flight before the MMAs of this one are issued and examined afterwards.
-template <int J, int NI, int PF_STAGES>
+template <int J, int NI, int PF_STAGES, int MT>
 __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, int n_mt, int* err) {
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
@@ -123,12 +124,12 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
     uint32_t alo[PF_STAGES], blo[PF_STAGES];
 #pragma unroll
     for (int s = 0; s < PF_STAGES; ++s) {
-        const uint32_t a = smem0 + (uint32_t)s * PF_STAGE_BYTES;
+        const uint32_t a = smem0 + (uint32_t)s * pf_stage_bytes(MT);
         alo[s] = (uint32_t)pf_smem_desc(a);
-        blo[s] = (uint32_t)pf_smem_desc(a + PF_MT * PF_ATOM_BYTES);
+        blo[s] = (uint32_t)pf_smem_desc(a + MT * PF_ATOM_BYTES);
     }
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
-    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BN * PF_MT);
+    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BN * MT);
     uint32_t ready = mbar_test(full(J), 0);
     uint32_t ph = 0;
     for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
@@ -143,7 +144,7 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
             if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int mt = 0; mt < PF_MT; ++mt)
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                 for (int ks = 0; ks < PF_BK / 16; ++ks)
                     if (mt < n_mt)
@@ -155,9 +156,12 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
     pf_commit(accum);  // this issuer's accumulators are complete once all its MMAs have finished
 }
 
-// PF_STAGES stages, NG producer groups (a stage buffer always belongs to the same group), NI issuers with their own
-// accumulators.  Instantiated as <bits, 4, 4, 2>.
-template <int BITS, int PF_STAGES, int NG, int NI>
+// PF_STAGES stages, NG producer groups (K block kb is decoded by group kb % NG into stage kb % PF_STAGES), NI issuers with
+// their own accumulators, MT token tiles of 128 per CTA.  Instantiated as <bits, 4, 4, 2, 2> (M > 128: 256-token tiles,
+// four 48 KB stages) and <bits, 6, 4, 2, 1> (M <= 128: one token tile, six 32 KB stages -- a stage buffer's round trip
+// producer -> issuer -> tensor pipe -> producer is ~2400 cycles whatever the tile holds, so more buffers = more stages
+// per unit of time).
+template <int BITS, int PF_STAGES, int NG, int NI, int MT>
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
@@ -166,7 +170,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * PF_STAGE_BYTES);
+    constexpr int STAGE_BYTES = pf_stage_bytes(MT);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PF_STAGES + 1);
     const uint32_t bar0 = smem_u32(bars);
@@ -176,8 +181,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
 
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
-    constexpr int TMEM_COLS = NI * PF_BN * PF_MT;       // one pair of accumulators per issuer
-    static_assert(PF_STAGES % NG == 0 && NG % 2 == 0 && PF_STAGES % NI == 0, "a stage buffer belongs to one group and one issuer");
+    constexpr int TMEM_COLS = NI * PF_BN * MT;          // MT accumulators per issuer
+    static_assert(NG % 2 == 0 && PF_STAGES % NI == 0, "a group always decodes the same half of a column block; a stage buffer belongs to one issuer");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
     // into tail_splits items along K, so that the last, partly filled wave of CTAs is short.  Tiles are numbered
@@ -194,7 +199,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     {
         int tile, zsplit, splits;
         item(tile, zsplit, splits);
-        m0 = (int64_t)(tile % tiles_m) * (PF_BM * PF_MT);
+        m0 = (int64_t)(tile % tiles_m) * (PF_BM * MT);
         n0 = (int64_t)(tile / tiles_m) * PF_BN;
         // split item z of a tile owns column blocks [cb0, cb1), two stages each
         cb0 = (int64_t)zsplit * (K / 128) / splits;
@@ -202,7 +207,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     }
     const int64_t ncb = K / 128;
     // a tile with at most 128 real tokens (decode batches, the ragged last token tile) uses one accumulator only
-    const int n_mt = M - m0 > PF_BM ? PF_MT : 1;
+    const int n_mt = M - m0 > PF_BM ? MT : 1;
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
@@ -233,18 +238,20 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
                 }
-                mbar_expect_tx(full(s), (uint32_t)n_mt * PF_ATOM_BYTES);
-                const uint32_t a = smem_u32(smem + (size_t)s * PF_STAGE_BYTES);
+                // MT == 1 (M <= 128): the box holds exactly the M token rows -- the TMA unit spends time on every row of a
+                // box, in range or not; the rows of the tile that nothing writes belong to tokens that are never stored
+                mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u : (uint32_t)n_mt * PF_ATOM_BYTES);
+                const uint32_t a = smem_u32(smem + (size_t)s * STAGE_BYTES);
 #pragma unroll
-                for (int mt = 0; mt < PF_MT; ++mt)
+                for (int mt = 0; mt < MT; ++mt)
                     if (mt < n_mt) pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
             }
         }
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
-            else pf_issue<NI - 1, NI, PF_STAGES>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
+            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
+            else pf_issue<NI - 1, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
         }
     } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
@@ -297,7 +304,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
                     __syncwarp();
                 }
-                unsigned char* brow = smem + (size_t)s * PF_STAGE_BYTES + PF_MT * PF_ATOM_BYTES + row * 128;
+                unsigned char* brow = smem + (size_t)s * STAGE_BYTES + MT * PF_ATOM_BYTES + row * 128;
                 const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
 #pragma unroll
                 for (int T2 = 0; T2 < 2; ++T2) {
@@ -327,14 +334,15 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
         const int ew = warp - PROD_WARP0;
-        const int mt = (ew >> 2) & 1;             // four warps per accumulator; with NG = 4 two sets of them share the columns
-        constexpr int CHUNKS = (PF_BN / 32) / (NG / 2);
-        const int cc0 = (ew >> 3) * CHUNKS;
+        // four warps (one per lane quarter) per accumulator; the NG / MT sets of them split the 128 columns
+        const int mt = MT == 2 ? (ew >> 2) & 1 : 0;
+        constexpr int CHUNKS = (PF_BN / 32) * MT / NG;
+        const int cc0 = (MT == 2 ? ew >> 3 : ew >> 2) * CHUNKS;
         const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
         int tile, zsplit, splits;  // recomputed here rather than kept in registers across the main loop
         item(tile, zsplit, splits);
         const int tail_index = tile - n_full;   // index of the tile among the split ones
-        const int64_t rows_alloc = M < PF_BM * PF_MT ? M : PF_BM * PF_MT;  // token rows kept per tile in the workspace
+        const int64_t rows_alloc = M < PF_BM * MT ? M : PF_BM * MT;  // token rows kept per tile in the workspace
         auto store_row = [&](const uint32_t (&v)[32], int col) {  // 32 FP32 sums of one token -> FP16 -> Y
             __half* dst = Y + token * N + n0 + col;
             if (n0 + col + 32 <= N) {
@@ -361,7 +369,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(mt * PF_BN + col), v);
             if (NI == 2) {                        // add the second issuer's sums (odd stages) to the first's: a fixed order
                 uint32_t v1[32];
-                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BN * PF_MT + mt * PF_BN + col), v1);
+                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BN * MT + mt * PF_BN + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
@@ -501,24 +509,29 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
     CUtensorMap xmap;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {64, PF_BM};
+    const cuuint32_t box[2] = {64, (cuuint32_t)(M <= PF_BM ? M : PF_BM)};  // M <= 128 runs the one-tile kernel: no padding rows
     const cuuint32_t estr[2] = {1, 1};
     if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
     const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits));
-    auto run = [&](auto kernel) -> pot_status_t {
-        const size_t smem = pf_smem_bytes(4);
+    auto run = [&](auto kernel, int stages, int mt) -> pot_status_t {
+        const size_t smem = pf_smem_bytes(stages, mt);
         const dim3 block((unsigned)pf_threads(4, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (__half*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
-    // four stages, four producer groups, two issuers: one CTA per SM
-    if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2>);
-    if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2>);
-    return run(pot_gemm_prefill_kernel<4, 4, 4, 2>);
+    // four producer groups, two issuers, one CTA per SM; one token tile and six stages for batches of up to 128 tokens
+    if (M <= PF_BM) {
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 4, 2, 1>, 6, 1);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 4, 2, 1>, 6, 1);
+        return run(pot_gemm_prefill_kernel<4, 6, 4, 2, 1>, 6, 1);
+    }
+    if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2>, 4, 2);
+    if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2>, 4, 2);
+    return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2>, 4, 2);
 }
 
 static int* prefill_error_ptr() { return ring_error_ptr(); }
