@@ -45,9 +45,11 @@ constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
 __host__ __device__ constexpr int pf_stage_bytes(int mt) { return (mt + 1) * PF_ATOM_BYTES; }
 constexpr size_t pf_smem_bytes(int stages, int mt) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt) + 256 /*barriers*/; }
 
-// UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
-constexpr uint32_t PF_IDESC = (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ |
-                              ((uint32_t)(PF_BN >> 3) << 17) | ((uint32_t)(PF_BM >> 4) << 24);
+// UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128 (the weight rows of the tile are the
+// A operand), N = n token rows of the X tile (the B operand), 16 <= n <= 256, n % 16 == 0
+__host__ __device__ constexpr uint32_t pf_idesc(uint32_t n) {
+    return (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ | ((n >> 3) << 17) | ((uint32_t)(PF_BN >> 4) << 24);
+}
 
 // shared-memory matrix descriptor, K-major, 128-byte swizzle: start >> 4, LBO = 1 (unused), SBO = 1024 B
 // between 8-row groups, descriptor version 1, layout type 2 (SWIZZLE_128B)
@@ -111,13 +113,13 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 
 // The MMA issuer J of NI (one thread): takes the stages kb = J, J + NI, ... of the CTA's nkb stages and accumulates them
-// into its own pair of accumulators.  One thread's dependent instructions retire every ~5 cycles and the tensor pipe
+// into its own accumulator (128 weight rows = lanes, n_tok token columns).  One thread's dependent instructions retire every ~5 cycles and the tensor pipe
 // idles meanwhile, so what the loop needs per MMA is prepared first: the low descriptor word of every stage's tiles (the
 // high word is a constant); the loop is unrolled over the stages so that these stay in registers and a K step is one
 // add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the test for the issuer's
 // next stage is put in flight before the MMAs of this one are issued and examined afterwards.
 template <int J, int NI, int PF_STAGES, int MT>
-__device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, int n_mt, int* err) {
+__device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, uint32_t n_tok, int* err) {
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
     const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
@@ -129,7 +131,8 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
         blo[s] = (uint32_t)pf_smem_desc(a + MT * PF_ATOM_BYTES);
     }
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
-    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BN * MT);
+    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BM * MT);   // this issuer's accumulator: 128 features x (128 MT) token columns
+    const uint32_t idesc = pf_idesc(n_tok);
     uint32_t ready = mbar_test(full(J), 0);
     uint32_t ph = 0;
     for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
@@ -144,12 +147,9 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
             if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int ks = 0; ks < PF_BK / 16; ++ks)
-                    if (mt < n_mt)
-                        pf_mma2(d0 + (uint32_t)(mt * PF_BN), alo[s] + (uint32_t)((mt * PF_ATOM_BYTES + ks * 32) >> 4),
-                                blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, PF_IDESC, (s != J || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
+            for (int ks = 0; ks < PF_BK / 16; ++ks)  // A = the decoded weight tile, B = the X tile(s): one MMA covers all tokens
+                pf_mma2(d0, blo[s] + (uint32_t)((ks * 32) >> 4), alo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, idesc,
+                        (s != J || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
             pf_commit(empty(s));  // the stage is free again once these MMAs have read it
         }
     }
@@ -208,6 +208,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const int64_t ncb = K / 128;
     // a tile with at most 128 real tokens (decode batches, the ragged last token tile) uses one accumulator only
     const int n_mt = M - m0 > PF_BM ? MT : 1;
+    // token rows the MMA reads from the X stage: whole tiles, or (one-tile kernel) the batch rounded up to the MMA's N step
+    const uint32_t n_tok = MT == 1 ? (uint32_t)((M + 15) & ~(int64_t)15) : (uint32_t)(n_mt * PF_BM);
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
@@ -250,8 +252,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
-            else pf_issue<NI - 1, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_mt, err);
+            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            else pf_issue<NI - 1, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
         }
     } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
@@ -332,58 +334,41 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (err) atomicCAS(err, 0, 0x40);
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int q = warp & 3;                   // this warp may only touch TMEM lanes 32q .. 32q+31
-        const int ew = warp - PROD_WARP0;
-        // four warps (one per lane quarter) per accumulator; the NG / MT sets of them split the 128 columns
-        const int mt = MT == 2 ? (ew >> 2) & 1 : 0;
-        constexpr int CHUNKS = (PF_BN / 32) * MT / NG;
-        const int cc0 = (MT == 2 ? ew >> 3 : ew >> 2) * CHUNKS;
-        const int64_t token = m0 + mt * PF_BM + 32 * q + lane;
+        // Lane = weight row (feature), column = token.  Warp (q, part): features n0 + 32 q .. + 31 (a warp may only touch its
+        // own quarter of the lanes), token columns part * 32 MT .. + 32 MT - 1.
+        const int q = warp & 3;
+        const int part = (warp - PROD_WARP0) >> 2;
+        const int64_t feat = n0 + 32 * q + lane;
         int tile, zsplit, splits;  // recomputed here rather than kept in registers across the main loop
         item(tile, zsplit, splits);
         const int tail_index = tile - n_full;   // index of the tile among the split ones
         const int64_t rows_alloc = M < PF_BM * MT ? M : PF_BM * MT;  // token rows kept per tile in the workspace
-        auto store_row = [&](const uint32_t (&v)[32], int col) {  // 32 FP32 sums of one token -> FP16 -> Y
-            __half* dst = Y + token * N + n0 + col;
-            if (n0 + col + 32 <= N) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    uint32_t o[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const __half2 h = __floats2half2_rn(__uint_as_float(v[8 * i + 2 * j]), __uint_as_float(v[8 * i + 2 * j + 1]));
-                        o[j] = *reinterpret_cast<const uint32_t*>(&h);
-                    }
-                    *reinterpret_cast<uint4*>(dst + 8 * i) = make_uint4(o[0], o[1], o[2], o[3]);
-                }
-            } else {
-                for (int i = 0; i < 32; ++i)
-                    if (n0 + col + i < N) dst[i] = __float2half_rn(__uint_as_float(v[i]));
-            }
-        };
-#pragma unroll
-        for (int cc = 0; cc < CHUNKS; ++cc) {
-            if (mt >= n_mt) break;                // (warp-uniform) no token of this accumulator exists
-            const int col = (cc0 + cc) * 32;
+        for (int cc = 0; cc < MT; ++cc) {
+            const int col = (part * MT + cc) * 32;
+            if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
-            pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(mt * PF_BN + col), v);
+            pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
             if (NI == 2) {                        // add the second issuer's sums (odd stages) to the first's: a fixed order
                 uint32_t v1[32];
-                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BN * MT + mt * PF_BN + col), v1);
+                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BM * MT + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
             } else {
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             }
-            if (token < M) {
-                if (splits == 1) {
-                    store_row(v, col);
-                } else {  // this split's partial sums: [tail tile][split][token of the tile][128 features] FP32
-                    float* dst = partial + (((int64_t)tail_index * splits + zsplit) * rows_alloc + (token - m0)) * PF_BN + col;
+            if (feat < N) {
+                if (splits == 1) {  // a warp stores 32 consecutive features (64 bytes) of one token at a time
+                    __half* dst = Y + (m0 + col) * N + feat;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    for (int i = 0; i < 32; ++i)
+                        if (m0 + col + i < M) dst[(int64_t)i * N] = __float2half_rn(__uint_as_float(v[i]));
+                } else {  // this split's partial sums: [tail tile][split][token of the tile][128 features] FP32
+                    float* dst = partial + (((int64_t)tail_index * splits + zsplit) * rows_alloc + col) * PF_BN + (32 * q + lane);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (m0 + col + i < M) dst[(int64_t)i * PF_BN] = __uint_as_float(v[i]);
                 }
             }
         }
