@@ -35,6 +35,7 @@ namespace pot {
 constexpr int PF_BM = 128;      // tokens per accumulator (MMA M)
 constexpr int PF_MT = 2;        // accumulators per CTA: 256 tokens share one decoded weight tile
 constexpr int PF_BN = 128;      // features per tile (MMA N)
+constexpr int PF_TMA2_MAX_TOKENS = 64;  // up to this batch size two threads issue the X copies
 constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte swizzle atom wide)
 // Warps: 0 = TMA, 1 .. NI = MMA issuers, then (from a warp index that is a multiple of 2 or 4, so that warp & 3 walks the
 // tensor-memory lane quarters in step) NG groups of four dequant / epilogue warps.
@@ -232,10 +233,14 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     pdl_launch_dependents();
     pdl_wait();
 
-    if (warp == 0) {
-        // ---------------- TMA producer: two X tiles (64 columns x 128 tokens each) per stage --------------
-        if (lane == 0) {
-            for (int kb = 0; kb < nkb; ++kb) {
+    if (warp == 0 || (NI == 2 && warp == 3)) {
+        // ---------------- TMA producers: MT X tiles (64 columns x 128 tokens each) per stage ----------------
+        // One thread needs ~600 cycles per stage (barrier wait, expect_tx, TMA instruction: three long latencies in a
+        // row), which paces batches of a few tokens; there warp 3 (idle next to two issuers) takes every other
+        // stage.  With big boxes the TMA unit is the slower part and a second thread only adds contention.
+        const int n_tma = (NI == 2 && MT == 1 && M <= PF_TMA2_MAX_TOKENS) ? 2 : 1;
+        if (lane == 0 && (warp == 0 || n_tma == 2)) {
+            for (int kb = warp == 0 ? 0 : 1; kb < nkb; kb += n_tma) {
                 const int s = kb % PF_STAGES;
                 if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
