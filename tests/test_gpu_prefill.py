@@ -1,4 +1,4 @@
-"""GPU parity: the tcgen05 prefill GEMM (tiled layout, M > 32) against the FP64 oracle."""
+"""GPU parity: the tcgen05 GEMM (tiled layout, M > 8) against the FP64 oracle."""
 import numpy as np
 import pytest
 
@@ -15,8 +15,12 @@ def B():
     return binding
 
 
-# (M, N, K): one exact tile; ragged M and N with several K blocks; several tiles in both directions
-SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20, 256, 4096)]  # the last two run split-K
+# (M, N, K).  M <= 128 runs the one-token-tile variant (six stages, a TMA box of exactly M rows; up to 64 tokens two
+# threads issue the X copies), larger M the 256-token tiles: one exact tile; ragged M and N with several K blocks; several
+# tiles in both directions; (300, ...) and (20, ...) run split-K; 129 tokens = a second token tile that holds one token;
+# K = 1152 / 2048 = more K blocks than pipeline stages
+SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20, 256, 4096), (129, 144, 640),
+          (64, 272, 1152), (9, 48, 2048), (65, 160, 1152)]
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -49,6 +53,19 @@ def test_split_k_workspace_is_reusable(B, oracle):
     assert np.array_equal(y1, y2)
     ok, worst, tight = gate(y1, Y, A)
     assert ok and tight < 4.0, (worst, tight)
+
+
+def test_two_issuers_give_the_same_bits_every_time(B, oracle):
+    """The two MMA issuers accumulate alternate K blocks into separate accumulators that the epilogue adds in a fixed
+    order: nothing in the result may depend on which of them ran first."""
+    bits, G, M, N, K = 3, 128, 300, 272, 2304
+    c = PotCase(N, K, bits, G, dist="t5", seed=(5, 88))
+    dX = f16_dev(synth.activations(synth.rng_for(5, 188), M, K, outliers=True))
+    ws = B.new_workspace(B.pot_gemm_workspace_bytes(M, N, K, bits, G))
+    y0 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
+    for _ in range(4):
+        assert np.array_equal(bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws)), y0)
+    assert B.pot_debug_errors() == (0, 0, 0)
 
 
 @pytest.mark.parametrize("bits", [3])
