@@ -7,18 +7,21 @@
 //   warps 4..19        : "dequant producers", four groups of four warps that take the stages in turn -- each thread
 //                        fetches the 32 codes of one weight row that the stage needs (8-byte loads from the tiled
 //                        layout, prefetched three of the group's stages ahead), decodes them in registers with the
-//                        mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the stage's B tile in
+//                        mask / shift-add trick of Sec. 4.2 and writes the FP16 values into the stage's weight tile in
 //                        exactly the layout the tensor core expects (K-major, 8-row x 128-byte atoms, 16-byte chunks
 //                        XOR-swizzled with the row index), then fence.proxy.async + mbarrier arrive;
-//   warps 1, 2 (one lane each) : the two MMA issuers take alternate stages; each waits for both operands, issues
-//                        2 x 4 tcgen05.mma (M = 128, N = 128, K = 16) into ITS OWN pair of 128-column accumulators
-//                        in tensor memory and tcgen05.commit's the stage back to the producers.  One issuing thread
-//                        leaves the tensor pipe idle for several hundred cycles per stage (barrier test, fence,
-//                        commit, the pipe's start-up after a gap); two threads fill each other's gaps.
+//   warps 1, 2 (one lane each) : the two MMA issuers take alternate stages; each waits for both operands, issues four
+//                        tcgen05.mma (A = the 128 decoded weight rows, B = the 256 tokens: M = 128, N = 256, K = 16) into
+//                        ITS OWN 256 columns of tensor memory (lane = weight row, column = token) and tcgen05.commit's
+//                        the stage back to the producers.  One issuing thread leaves the tensor pipe idle for several
+//                        hundred cycles per stage (barrier test, fence, commit, the pipe's start-up after a gap); two
+//                        threads fill each other's gaps.
 // After the last K block each issuer commits to a common barrier; the producer warps read the accumulators with
 // tcgen05.ld (each warp its own 32-lane quarter), add the two issuers' sums in a fixed order, convert to FP16 and
-// store.  The weights are re-decoded once per 256-token tile (M / 256 times overall), which is the price of never
-// writing FP16 weights to HBM.  A tile with at most 128 real tokens uses one accumulator per issuer only.
+// store (a warp writes 32 consecutive features of one token at a time).  The weights are re-decoded once per 256-token
+// tile (M / 256 times overall), which is the price of never writing FP16 weights to HBM.
+// Batches of up to 64 tokens run a variant with one tile of M token rows (the TMA box holds exactly M rows, the MMA's
+// N is M rounded up to 16), eight 24 KB stages and two TMA threads.
 //
 // All mbarrier waits are bounded (see ring.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
@@ -35,7 +38,7 @@ namespace pot {
 constexpr int PF_BM = 128;      // tokens per accumulator (MMA M)
 constexpr int PF_MT = 2;        // accumulators per CTA: 256 tokens share one decoded weight tile
 constexpr int PF_BN = 128;      // features per tile (MMA N)
-constexpr int PF_TMA2_MAX_TOKENS = 64;  // up to this batch size two threads issue the X copies
+constexpr int PF_SMALL_TOKENS = 64;     // largest batch of the one-token-tile kernel (its X stage holds 64 rows)
 constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte swizzle atom wide)
 // Warps: 0 = TMA, 1 .. NI = MMA issuers, then (from a warp index that is a multiple of 2 or 4, so that warp & 3 walks the
 // tensor-memory lane quarters in step) NG groups of four dequant / epilogue warps.
@@ -43,7 +46,9 @@ __host__ __device__ constexpr int pf_prod_warp0(int ni) { return ni == 2 ? 4 : 2
 __host__ __device__ constexpr int pf_threads(int ng, int ni) { return (pf_prod_warp0(ni) + 4 * ng) * 32; }
 constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
 // a stage: MT X tiles (token tiles) + one weight tile
-__host__ __device__ constexpr int pf_stage_bytes(int mt) { return (mt + 1) * PF_ATOM_BYTES; }
+// (the one-tile kernel serves up to PF_SMALL_TOKENS tokens: 8 KB of X per stage, so that eight stages fit)
+__host__ __device__ constexpr int pf_x_bytes(int mt) { return mt == 1 ? PF_SMALL_TOKENS * 128 : mt * PF_ATOM_BYTES; }
+__host__ __device__ constexpr int pf_stage_bytes(int mt) { return pf_x_bytes(mt) + PF_ATOM_BYTES; }
 constexpr size_t pf_smem_bytes(int stages, int mt) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt) + 256 /*barriers*/; }
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128 (the weight rows of the tile are the
@@ -129,7 +134,7 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
     for (int s = 0; s < PF_STAGES; ++s) {
         const uint32_t a = smem0 + (uint32_t)s * pf_stage_bytes(MT);
         alo[s] = (uint32_t)pf_smem_desc(a);
-        blo[s] = (uint32_t)pf_smem_desc(a + MT * PF_ATOM_BYTES);
+        blo[s] = (uint32_t)pf_smem_desc(a + pf_x_bytes(MT));
     }
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
     const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BM * MT);   // this issuer's accumulator: 128 features x (128 MT) token columns
@@ -158,10 +163,12 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
 }
 
 // PF_STAGES stages, NG producer groups (K block kb is decoded by group kb % NG into stage kb % PF_STAGES), NI issuers with
-// their own accumulators, MT token tiles of 128 per CTA.  Instantiated as <bits, 4, 4, 2, 2> (M > 128: 256-token tiles,
-// four 48 KB stages) and <bits, 6, 4, 2, 1> (M <= 128: one token tile, six 32 KB stages -- a stage buffer's round trip
-// producer -> issuer -> tensor pipe -> producer is ~2400 cycles whatever the tile holds, so more buffers = more stages
-// per unit of time).
+// their own accumulators, MT token tiles of 128 per CTA.  PF_STAGES is a multiple of NG and of NI: a stage buffer is
+// always filled by the same group, loaded by the same TMA thread and read by the same issuer, so every parity wait is
+// made by a thread that has itself seen the barrier's previous phase (a waiter two phases behind could not tell).
+// Instantiated as <bits, 4, 4, 2, 2> (M > 64: 256-token tiles, four 48 KB stages) and <bits, 8, 4, 2, 1> (M <= 64: one
+// tile of up to 64 tokens, eight 24 KB stages -- a stage buffer's round trip producer -> issuer -> tensor pipe ->
+// producer is ~2000 cycles whatever the tile holds, so more buffers = more stages per unit of time).
 template <int BITS, int PF_STAGES, int NG, int NI, int MT>
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
@@ -183,7 +190,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
     constexpr int TMEM_COLS = NI * PF_BN * MT;          // MT accumulators per issuer
-    static_assert(NG % 2 == 0 && PF_STAGES % NI == 0, "a group always decodes the same half of a column block; a stage buffer belongs to one issuer");
+    static_assert(NG % 2 == 0 && PF_STAGES % NI == 0 && PF_STAGES % NG == 0,
+                  "a group always decodes the same half of a column block; a stage buffer belongs to one issuer and one group");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
     // into tail_splits items along K, so that the last, partly filled wave of CTAs is short.  Tiles are numbered
@@ -210,7 +218,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     // a tile with at most 128 real tokens (decode batches, the ragged last token tile) uses one accumulator only
     const int n_mt = M - m0 > PF_BM ? MT : 1;
     // token rows the MMA reads from the X stage: whole tiles, or (one-tile kernel) the batch rounded up to the MMA's N step
-    const uint32_t n_tok = MT == 1 ? (uint32_t)((M + 15) & ~(int64_t)15) : (uint32_t)(n_mt * PF_BM);
+    const uint32_t n_tok = MT == 1 ? (uint32_t)((M + 15) & ~(int64_t)15) : (uint32_t)(n_mt * PF_BM);  // MT == 1: M <= 64
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
@@ -238,14 +246,17 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         // One thread needs ~600 cycles per stage (barrier wait, expect_tx, TMA instruction: three long latencies in a
         // row), which paces batches of a few tokens; there warp 3 (idle next to two issuers) takes every other
         // stage.  With big boxes the TMA unit is the slower part and a second thread only adds contention.
-        const int n_tma = (NI == 2 && MT == 1 && M <= PF_TMA2_MAX_TOKENS) ? 2 : 1;
+        const int n_tma = (NI == 2 && MT == 1) ? 2 : 1;
         if (lane == 0 && (warp == 0 || n_tma == 2)) {
+            uint32_t ready = 0;  // the test of the next stage's barrier is in flight while this stage's copies are issued
             for (int kb = warp == 0 ? 0 : 1; kb < nkb; kb += n_tma) {
                 const int s = kb % PF_STAGES;
-                if (kb >= PF_STAGES && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
+                if (kb >= PF_STAGES && !ready && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
                 }
-                // MT == 1 (M <= 128): the box holds exactly the M token rows -- the TMA unit spends time on every row of a
+                const int kn = kb + n_tma;
+                ready = (kn < nkb && kn >= PF_STAGES) ? mbar_test(empty(kn % PF_STAGES), (uint32_t)((kn / PF_STAGES - 1) & 1)) : 0u;
+                // MT == 1 (M <= 64): the box holds exactly the M token rows -- the TMA unit spends time on every row of a
                 // box, in range or not; the rows of the tile that nothing writes belong to tokens that are never stored
                 mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u : (uint32_t)n_mt * PF_ATOM_BYTES);
                 const uint32_t a = smem_u32(smem + (size_t)s * STAGE_BYTES);
@@ -311,7 +322,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
                     __syncwarp();
                 }
-                unsigned char* brow = smem + (size_t)s * STAGE_BYTES + MT * PF_ATOM_BYTES + row * 128;
+                unsigned char* brow = smem + (size_t)s * STAGE_BYTES + pf_x_bytes(MT) + row * 128;
                 const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
 #pragma unroll
                 for (int T2 = 0; T2 < 2; ++T2) {
@@ -354,7 +365,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
-            if (NI == 2) {                        // add the second issuer's sums (odd stages) to the first's: a fixed order
+            if (NI == 2) {                        // add the second issuer's sums (odd K blocks) to the first's: a fixed order
                 uint32_t v1[32];
                 pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BM * MT + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -499,7 +510,7 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
     CUtensorMap xmap;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)(M <= PF_BM ? M : PF_BM)};  // M <= 128 runs the one-tile kernel: no padding rows
+    const cuuint32_t box[2] = {64, (cuuint32_t)(M <= PF_SMALL_TOKENS ? M : PF_BM)};  // the one-tile kernel: no padding rows
     const cuuint32_t estr[2] = {1, 1};
     if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -513,11 +524,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (__half*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
-    // four producer groups, two issuers, one CTA per SM; one token tile and six stages for batches of up to 128 tokens
-    if (M <= PF_BM) {
-        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 4, 2, 1>, 6, 1);
-        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 4, 2, 1>, 6, 1);
-        return run(pot_gemm_prefill_kernel<4, 6, 4, 2, 1>, 6, 1);
+    // four producer groups, two issuers, one CTA per SM; one token tile and eight 24 KB stages for batches of up to 64 tokens
+    if (M <= PF_SMALL_TOKENS) {
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1>, 8, 1);
+        return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1>, 8, 1);
     }
     if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2>, 4, 2);
     if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2>, 4, 2);

@@ -15,10 +15,10 @@ def B():
     return binding
 
 
-# (M, N, K).  M <= 128 runs the one-token-tile variant (six stages, a TMA box of exactly M rows; up to 64 tokens two
-# threads issue the X copies), larger M the 256-token tiles: one exact tile; ragged M and N with several K blocks; several
-# tiles in both directions; (300, ...) and (20, ...) run split-K; 129 tokens = a second token tile that holds one token;
-# K = 1152 / 2048 = more K blocks than pipeline stages
+# (M, N, K).  M <= 64 runs the one-token-tile variant (eight stages, a TMA box of exactly M rows, two TMA threads), larger
+# M the 256-token tiles: one exact tile; ragged M and N with several K blocks; several tiles in both directions;
+# (300, ...) and (20, ...) run split-K; 129 tokens = a second token tile that holds one token; 64 / 65 tokens = either
+# side of the variant boundary; K = 1152 / 2048 = more K blocks than pipeline stages
 SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20, 256, 4096), (129, 144, 640),
           (64, 272, 1152), (9, 48, 2048), (65, 160, 1152)]
 
