@@ -235,9 +235,11 @@ pot_status_t pot_gemv_chain_run(const void* scratch, int n_ops, int bits, void* 
  * accumulation, FP16 output.  M <= 8 (decode batches) runs a bandwidth-bound tensor-core
  * kernel that decodes weights straight into MMA fragments; larger M (prefill) runs the
  * tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
- * accumulators in tensor memory; when the output tiles cover less than half of the SMs it
- * splits K across CTAs (FP32 partial sums and arrival counters in `workspace`, added in a fixed
- * order).  The tcgen05 kernel requires layout == POT_LAYOUT_TILED.
+ * accumulators in tensor memory (two issuing threads with an accumulator each, added in a fixed
+ * order: the result does not depend on timing); the tiles of a last, at most half-filled wave
+ * of CTAs -- or all tiles when they cover at most half of the SMs -- are split along K (FP32
+ * partial sums and arrival counters in `workspace`, added in a fixed order).  The tcgen05
+ * kernel requires layout == POT_LAYOUT_TILED.
  *   workspace >= pot_gemm_workspace_bytes(M,N,K,bits,group), 16-byte aligned, zero before its
  *   first use (the kernels leave the counters at zero); may be NULL when that size is 0.
  */
