@@ -35,9 +35,9 @@
 
 namespace pot {
 
-constexpr int PF_BM = 128;      // tokens per accumulator (MMA M)
-constexpr int PF_MT = 2;        // accumulators per CTA: 256 tokens share one decoded weight tile
-constexpr int PF_BN = 128;      // features per tile (MMA N)
+constexpr int PF_BM = 128;      // tokens per X tile (TMA box rows; one MMA covers one or two of them as its N side)
+constexpr int PF_MT = 2;        // X tiles per CTA of the large-M kernel: 256 tokens share one decoded weight tile
+constexpr int PF_BN = 128;      // features (weight rows) per tile: the MMA's M side, the accumulator's lanes
 constexpr int PF_SMALL_TOKENS = 64;     // largest batch of the one-token-tile kernel (its X stage holds 64 rows)
 constexpr int PF_BK = 64;       // half a column block per stage (one 128-byte swizzle atom wide)
 // Warps: 0 = TMA, 1 .. NI = MMA issuers, then (from a warp index that is a multiple of 2 or 4, so that warp & 3 walks the
@@ -72,15 +72,7 @@ __device__ __forceinline__ void pf_tma_load_2d(uint32_t dst, const CUtensorMap* 
                  "l"(map), "r"(x), "r"(y), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void pf_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// same, the two descriptors given as their low words + the common high word
+// tcgen05.mma, the two operand descriptors given as their low words + the common high word
 __device__ __forceinline__ void pf_mma2(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
