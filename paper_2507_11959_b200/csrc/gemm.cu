@@ -1,6 +1,7 @@
 // pot_gemm: Y[M,N] = X[M,K] W~^T with the dequantization fused in.
 //
-//  * M <= 8, tiled layout: bandwidth-bound tensor-core kernel (ring.cuh).  The weights are the MMA's
+//  * M <= 6 (and 7, 8 where the tcgen05 kernel's tiles would fill the SMs badly), tiled layout: tensor-core kernel on
+//    the shared-memory ring (ring.cuh).  The weights are the MMA's
 //    M-side operand (16 rows per warp-step), the tokens its 8-wide N side, so no padding of M
 //    to 16 is needed and a warp decodes each record exactly once, straight into the A
 //    fragment registers -- the FP16 weights never exist in shared or global memory.
@@ -9,7 +10,7 @@
 //    gid+8, column block 4*chunk + tig) into k-slots {2tig, 2tig+1, 2tig+8, 2tig+9} of step j,
 //    and the B fragment reads x at the same columns.
 //  * any M, canonical layout: a plain shared-memory tiled mma.sync kernel (the fallback).
-//  * M > 8, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
+//  * otherwise, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
 #include "common.cuh"
 #include "layout.cuh"
 #include "ring.cuh"
@@ -112,23 +113,28 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s);
 size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int bits, int group);
 bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group);
+double gemm_prefill_wave_fill(int64_t M, int64_t N, int64_t K);
 
 }  // namespace pot
 
 using namespace pot;
 
-// Up to 8 tokens the streaming kernel (weights decoded straight into MMA fragments) is bandwidth-bound;
-// beyond that the legacy warp-level MMA rate becomes the limit and the tcgen05 kernel takes over.
-constexpr int64_t kSmallBatchMax = 8;
-static bool use_small(int64_t M, int64_t N, pot_layout_t layout) {
-    return layout == POT_LAYOUT_TILED && M <= kSmallBatchMax && N % 16 == 0;
+// The streaming kernel (weights decoded straight into MMA fragments) serves up to 8 tokens and its time grows with
+// the batch; the tcgen05 kernel's time is flat in the batch but has a higher floor and works in 128-feature tiles.
+// Measured cross-over: up to 6 tokens the streaming kernel wins everywhere; at 7 and 8 tokens the tcgen05 kernel wins
+// (by 15 - 25 %) unless its tiles fill the SMs badly (e.g. 86 or 96 tiles on 148 SMs: 10 % slower).
+constexpr int64_t kSmallBatchMax = 8, kSmallBatchAlways = 6;
+constexpr double kMinWaveFill = 0.75;
+static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout) {
+    if (layout != POT_LAYOUT_TILED || M > kSmallBatchMax || N % 16 != 0) return false;
+    return M <= kSmallBatchAlways || gemm_prefill_wave_fill(M, N, K) < kMinWaveFill;
 }
 
 static int small_mt(int64_t) { return 1; }
 
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || M <= 0) return 0;
-    if (M <= kSmallBatchMax && N % 16 == 0) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
+    if (use_small(M, N, K, POT_LAYOUT_TILED)) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
@@ -144,7 +150,7 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
     if (!aligned16(packed) || !aligned16(scales) || !aligned16(X) || !aligned16(Y) || !aligned16(workspace))
         return POT_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;
-    if (use_small(M, N, layout)) {
+    if (use_small(M, N, K, layout)) {
         const size_t need = pot_gemm_workspace_bytes(M, N, K, bits, group);
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
         const int Mi = (int)M;

@@ -45,8 +45,11 @@ def test_size_helpers(L):
     assert L.pot_gemv_workspace_bytes(12288, 512, 3, 128) == 0
     ws = L.pot_gemv_workspace_bytes(4096, 11008, 3, 128)
     assert ws == 1024 + 256 * 22 * 16 * 4 and ws % 16 == 0
-    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
-    # M > 8 runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
+    assert L.pot_gemm_workspace_bytes(6, 4096, 11008, 3, 128) == 1024 + 256 * 22 * 16 * 8 * 4
+    # 7 and 8 tokens: the streaming kernel only where the tcgen05 kernel's tiles would fill the SMs badly (96 tiles on 148)
+    assert L.pot_gemm_workspace_bytes(8, 12288, 4096, 3, 128) == L.pot_gemm_workspace_bytes(6, 12288, 4096, 3, 128)
+    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 256 + 32 * 4 * 8 * 128 * 4
+    # Larger M runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
     # cover at most half of the SMs (32 tiles -> 4 splits of 32 token rows x 128 features), or those of a last
     # wave that fills at most half of the 148 CTA slots (640 tiles -> 48 tail tiles x 3 splits x 256 rows).
     assert L.pot_gemm_workspace_bytes(32, 4096, 11008, 3, 128) == 256 + 32 * 4 * 32 * 128 * 4
