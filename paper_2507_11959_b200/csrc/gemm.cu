@@ -124,7 +124,7 @@ using namespace pot;
 // Measured cross-over: up to 6 tokens the streaming kernel wins everywhere; at 7 and 8 tokens the tcgen05 kernel wins
 // (by 15 - 25 %) unless its tiles fill the SMs badly (e.g. 86 or 96 tiles on 148 SMs: 10 % slower).
 constexpr int64_t kSmallBatchMax = 8, kSmallBatchAlways = 6;
-constexpr double kMinWaveFill = 0.75;
+constexpr double kMinWaveFill = 0.70;
 static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout) {
     if (layout != POT_LAYOUT_TILED || M > kSmallBatchMax || N % 16 != 0) return false;
     return M <= kSmallBatchAlways || gemm_prefill_wave_fill(M, N, K) < kMinWaveFill;
