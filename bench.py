@@ -189,6 +189,7 @@ def main():
             W = f16(synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5"))
             packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
             tiled = B.pot_repack(packed, pr.K, bits, 0)
+            S = B.pot_repack_scales(S, pr.K, GROUP, 0)
             x = f16(synth.activations(synth.rng_for(2, 2 * i + 1), 1, pr.K)[0])
             y = torch.empty(pr.N, dtype=torch.float16, device=dev)
             ws_bytes = B.pot_gemv_workspace_bytes(pr.N, pr.K, bits, GROUP)
@@ -423,28 +424,6 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
     del g2, layers2
     torch.cuda.empty_cache()
 
-    # the headline chain through pot_gemv_chain: one persistent cooperative kernel per step instead of a graph of
-    # 160 programmatically chained launches
-    layersc, bytesc = build_chain(HEADLINE_BITS)
-    ops = [(t, sc, pr.K, GROUP, x, y, ws) for layer in layersc for (pr, t, sc, x, y, ws) in layer]
-    scratch = B.pot_gemv_chain_prepare(ops, HEADLINE_BITS, stream)
-    with torch.cuda.stream(stream):
-        for _ in range(3):
-            B.pot_gemv_chain_run(scratch, len(ops), HEADLINE_BITS, stream)
-        stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(5, args.steps // 2)
-        e0.record(stream)
-        for _ in range(reps):
-            B.pot_gemv_chain_run(scratch, len(ops), HEADLINE_BITS, stream)
-        e1.record(stream)
-        stream.synchronize()
-    msc = e0.elapsed_time(e1) / reps
-    ex["chain_3bit_one_persistent_kernel"] = {"GBps": bytesc / msc / 1e6, "ms_per_step": msc,
-                                              "frac_of_measured_hbm": bytesc / msc / 1e6 / hbm, "launches_per_step": 1}
-    del scratch, ops, layersc
-    torch.cuda.empty_cache()
-
     # the same 3-bit chain with gate and up stored as one 4096 -> 22016 matrix (they share their input, as qkv do):
     # 128 launches per step instead of 160 over the same weights
     fused = (synth.LLAMA2_7B[0], synth.LLAMA2_7B[1], synth.Projection("gate_up", 4096, 22016), synth.LLAMA2_7B[4])
@@ -469,8 +448,10 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
         for bits in (2, 3, 4):
             packed, S = B.pot_quantize_ref(W, bits, GROUP, B.SCALE_TOP)
             tiled = B.pot_repack(packed, K, bits, 0)
+            S = B.pot_repack_scales(S, K, GROUP, 0)
             up, uS, uZ = B.uint_quantize_ref(W, bits, GROUP)
             utiled = B.uint_repack(up, K, bits, 0)
+            uS, uZ = B.pot_repack_scales(uS, K, GROUP, 0), B.pot_repack_scales(uZ, K, GROUP, 0)
             copies = max(2, int(4 * 126e6 / (N * K * bits / 8)) + 1)
             ws = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, bits, GROUP), dev)
             pts = [(tiled.clone(), S.clone()) for _ in range(copies)]
@@ -517,6 +498,7 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
         W = f16(synth.weights(synth.rng_for(4, pr.N % 83), pr.N, pr.K, "t5"))
         packed, S = B.pot_quantize_ref(W, 3, GROUP, B.SCALE_TOP)
         tiled = B.pot_repack(packed, pr.K, 3, 0)
+        S = B.pot_repack_scales(S, pr.K, GROUP, 0)
         copies = max(2, int(4 * 126e6 / (pr.N * pr.K * 3 / 8)) + 1)
         pts = [(tiled.clone(), S.clone()) for _ in range(copies)]
         del W, packed
@@ -544,11 +526,12 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
             layout, P = B.CANONICAL, packed
             try:
                 tiled = B.pot_repack(packed, pr.K, bits, 0)
+                Sc, S = S, B.pot_repack_scales(S, pr.K, GROUP, 0)
                 ws = B.new_workspace(B.pot_gemm_workspace_bytes(synth.PREFILL_M, pr.N, pr.K, bits, GROUP), dev)
                 B.pot_gemm(tiled, S, pr.K, bits, GROUP, X, B.TILED, Y=Y, workspace=ws, stream=stream)
                 layout, P = B.TILED, tiled
             except B.PotError:
-                ws = None
+                ws, S = None, Sc
             g = capture(lambda s: B.pot_gemm(P, S, pr.K, bits, GROUP, X, layout, Y=Y, workspace=ws, stream=s))
             t = min(time_graph(g, 3, 3) for _ in range(2))
             fl = 2.0 * synth.PREFILL_M * pr.N * pr.K

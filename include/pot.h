@@ -79,10 +79,13 @@ const char* pot_status_string(pot_status_t s);
 /* ---- sizes (host arithmetic only; 0 on invalid arguments) ------------------------------- */
 size_t pot_packed_bytes(int64_t N, int64_t K, int bits);          /* N * K * bits / 8          */
 size_t pot_scales_bytes(int64_t N, int64_t K, int group);         /* N * (K / group) * 2       */
-/* Scratch needed by pot_gemv / uint_gemv with the tiled layout (split-K arrival counters +
- * FP32 partial sums); may be 0.  The workspace must be ZERO before its first use; every call
- * leaves the counters at zero again, so one buffer can serve all calls on one stream.  Two
- * calls that may run concurrently (different streams) need different workspaces.            */
+/* Scratch needed by pot_gemv / uint_gemv with the tiled layout (arrival counters of the row
+ * blocks + FP32 partial sums); may be 0.  The workspace must be ZERO before its first use; every
+ * call leaves its counters at zero again, so consecutive calls of the SAME entry point with the
+ * SAME (N, K, bits, group) may reuse one buffer without clearing it.  The position of the
+ * counters inside the buffer depends on the shape: a buffer handed to a call with another shape
+ * (or to pot_gemm) must be cleared to zero first.  Two calls that may run concurrently
+ * (different streams) need different workspaces.                                              */
 size_t pot_gemv_workspace_bytes(int64_t N, int64_t K, int bits, int group);
 /* Scratch needed by pot_gemm for the given M; may be 0.                                       */
 size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group);
@@ -110,7 +113,10 @@ pot_status_t pot_quantize_ref(const void* W_f16, int64_t N, int64_t K, int bits,
                               pot_scale_rule_t rule, void* scales_f16, void* packed_out, void* stream);
 
 /*
- * pot_validate_scales -- counts scales outside the scale contract.
+ * pot_validate_scales -- counts scales outside the scale contract: the integer add of Sec. 4.2 equals the
+ * multiplication by 2^E of Eq. 1 only for normal FP16 scales whose exponent field e satisfies 1 <= e and
+ * e + q_max <= 30 (the paper does not discuss zero, subnormal or overflowing scales).  A caller that gets a non-zero
+ * count should treat its scales as POT_ERR_SCALE_RANGE.
  *   d_bad_count: device int32; the kernel ADDS the number of offending entries (zero it first).
  */
 pot_status_t pot_validate_scales(const void* scales_f16, int64_t count, int bits, int32_t* d_bad_count,
@@ -133,6 +139,22 @@ pot_status_t pot_validate_scales(const void* scales_f16, int64_t count, int bits
 pot_status_t pot_repack(const void* src, void* dst, int64_t N, int64_t K, int bits, int direction,
                         void* stream);
 
+/*
+ * pot_repack_scales -- per-group parameters (the FP16 scales; also the uniform twin's zero-points) between the
+ * row-major [N, K/G] interchange layout and the tiled layout that goes with pot_repack (direction 0: row-major ->
+ * tiled, 1: back).  Same bytes, same size, N % 16 == 0; the buffers must not overlap.  (The paper fixes no storage
+ * order for the scales of Sec. 3.1; this one is the library's.)  The 16 * (128 / G) parameters of one unit are
+ * stored together, units in [rb][cb] order like the codes, so a kernel that streams a contiguous range of units
+ * fetches their scales with the same kind of contiguous copy; inside a unit the values of rows r and r + 8 of a
+ * group share a 32-bit word (halfword index ((s * 8 + r % 8) * 2 + r / 8) for group s of the unit).
+ * EVERY entry point that takes `layout == POT_LAYOUT_TILED` expects both the codes (pot_repack / uint_repack) and
+ * the per-group parameters (pot_repack_scales) in tiled form.
+ */
+pot_status_t pot_repack_scales(const void* src, void* dst, int64_t N, int64_t K, int group, int direction,
+                               void* stream);
+/* Host arithmetic only: halfword index, inside the tiled parameter array, of the value of (row, group g of the row). */
+pot_status_t pot_layout_scale_index(int64_t N, int64_t K, int group, int64_t row, int64_t g, int64_t* index);
+
 /* Host arithmetic only: position (32-bit word index inside the 4n-word record, bit index) of
  * bit b of code q (0 <= q < 128) in the tiled layout.  kind 0 = PoT codes, 1 = uniform codes. */
 pot_status_t pot_layout_bit(int bits, int kind, int q, int b, int* word, int* bit);
@@ -150,11 +172,12 @@ pot_status_t pot_dequant(const void* packed, const void* scales_f16, int64_t N, 
 /*
  * pot_gemv -- batch-1 decode: y = W~ x with W~ the FP16 reconstruction (Eq. 1), FP32
  * accumulation, FP16 output.  Codes are decoded in registers with the integer-add trick (Sec.
- * 4.2).  Tiled layout: a persistent kernel streams the codes through a shared-memory ring, the
- * decoded FP16 weights are the A fragments of warp-level tensor-core MMAs whose B columns all
- * hold x, and the matrix is split evenly across the SMs (partial sums of a row block that spans
- * CTAs go through `workspace` and are added in a fixed order, so results are bit-identical run
- * to run).  Canonical layout: a CUDA-core kernel with warp-shuffle reduction.
+ * 4.2).  Tiled layout: every warp streams its own contiguous share of the codes and scales
+ * through a private shared-memory ring, the decoded FP16 weights are the A fragments of
+ * warp-level tensor-core MMAs whose B columns all hold x, and the matrix is split evenly across
+ * all warps of the GPU (partial sums of a row block that spans warps are added in a fixed order --
+ * in shared memory inside a CTA, through `workspace` across CTAs -- so results are bit-identical
+ * run to run).  Canonical layout: a CUDA-core kernel with warp-shuffle reduction.
  *   x_f16 [K], y_f16 [N]; workspace >= pot_gemv_workspace_bytes(N,K,bits,group), 16-byte aligned
  *   (may be NULL when that size is 0).  `layout` says how `packed` is arranged.
  */
@@ -197,41 +220,8 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
                               int bits, int group, const void* x_f16, void* y_f16, void* stream);
 
 /*
- * pot_gemv_chain_* -- a list of dependent pot_gemv operations (tiled layout, one `bits` for the
- * whole list) executed by ONE persistent kernel instead of one launch per operation: between
- * two decode GEMVs of a few microseconds, the end-of-grid / start-of-grid latency of separate
- * launches costs as much as the arithmetic.  The kernel's CTAs stay resident, stream the next
- * operation's weights while the current one finishes, and meet at a grid-wide arrival counter
- * before they read the next activations, so operation i may read what operations < i wrote
- * (y of one as x of the next).  The paper has no counterpart; the arithmetic and the result of
- * every operation are those of pot_gemv (bit-identical).
- *   - pot_gemv_chain_prepare checks every operation (as pot_gemv does), writes the list into
- *     `scratch` (device memory, >= pot_gemv_chain_scratch_bytes(n_ops), 16-byte aligned) and zeroes
- *     the kernel's counters there; call it once per list, outside of stream capture.  The ops
- *     array is host memory and may be freed after the call returns.  POT_ERR_UNSUPPORTED when an
- *     operation's K exceeds 32768 (its activations must fit the kernel's shared memory).
- *   - pot_gemv_chain_run launches the kernel (cooperatively: all CTAs resident) on `stream`; it
- *     may be called any number of times after one prepare, with the same n_ops and bits.  Each
- *     operation's workspace must be zero before the first run (the kernel leaves it zero), and
- *     two operations may share a workspace.  Runs of one scratch must not overlap.
- */
-typedef struct {
-    const void* packed_tiled;   /* device, tiled layout                                   */
-    const void* scales_f16;     /* device [N, K/group]                                    */
-    int64_t N, K;
-    int group;
-    const void* x_f16;          /* device [K]                                             */
-    void* y_f16;                /* device [N]                                             */
-    void* workspace;            /* device, >= pot_gemv_workspace_bytes(N,K,bits,group)    */
-    size_t workspace_bytes;
-} pot_gemv_op_t;
-size_t pot_gemv_chain_scratch_bytes(int n_ops);
-pot_status_t pot_gemv_chain_prepare(const pot_gemv_op_t* ops_host, int n_ops, int bits, void* scratch,
-                                    size_t scratch_bytes, void* stream);
-pot_status_t pot_gemv_chain_run(const void* scratch, int n_ops, int bits, void* stream);
-
-/*
- * pot_gemm -- Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
+ * pot_gemm -- the matrix product that the dequantized weights feed (Sec. 4.2, last paragraph; reconstruction by
+ * Eq. 1, decode by the integer add of Sec. 4.2): Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
  * accumulation, FP16 output.  M <= 6 (decode batches; also M = 7, 8 on shapes whose 128-row
  * tiles would fill the SMs badly) runs a tensor-core kernel that decodes weights straight into
  * MMA fragments; larger M runs the tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,

@@ -22,10 +22,9 @@ UINT_FAST, UINT_NAIVE = 0, 1
 
 EXPORTS = [
     "pot_status_string", "pot_packed_bytes", "pot_scales_bytes", "pot_gemv_workspace_bytes",
-    "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack",
+    "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack", "pot_repack_scales", "pot_layout_scale_index",
     "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_host", "pot_gemm", "uint_quantize_ref", "uint_dequant",
-    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_gemv_chain_scratch_bytes", "pot_gemv_chain_prepare",
-    "pot_gemv_chain_run", "pot_debug_gemv_error", "pot_debug_gemm_error", "pot_debug_prefill_error",
+    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemm_error", "pot_debug_prefill_error",
 ]
 
 _lib = None
@@ -59,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.pot_validate_scales.argtypes = [vp, i64, i32, vp, vp]
         L.pot_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.uint_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
+        L.pot_repack_scales.argtypes = [vp, vp, i64, i64, i32, i32, vp]
+        L.pot_layout_scale_index.argtypes = [i64, i64, i32, i64, i64, vp]
         L.pot_dequant.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.pot_gemv.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
         L.pot_gemv_host.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -70,10 +71,6 @@ def lib() -> ctypes.CDLL:
         L.pot_gemv_noalloc.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp, vp]
         L.pot_gemv_noalloc_max_scratch_bytes.restype = sz
         L.pot_gemv_noalloc_max_scratch_bytes.argtypes = []
-        L.pot_gemv_chain_scratch_bytes.restype = sz
-        L.pot_gemv_chain_scratch_bytes.argtypes = [i32]
-        L.pot_gemv_chain_prepare.argtypes = [vp, i32, i32, vp, sz, vp]
-        L.pot_gemv_chain_run.argtypes = [vp, i32, i32, vp]
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is ctypes.c_int and name not in ("pot_status_string",):
@@ -159,6 +156,21 @@ def pot_repack(packed: torch.Tensor, K: int, bits: int, direction: int = 0, stre
     out = torch.empty_like(packed)
     _check(lib().pot_repack(_ptr(packed), _ptr(out), packed.shape[0], K, bits, direction, _stream(stream)), "pot_repack")
     return out
+
+
+def pot_repack_scales(scales: torch.Tensor, K: int, group: int, direction: int = 0, stream=None) -> torch.Tensor:
+    """Per-group parameters (scales, or the uniform twin's zero-points) [N, K/group]: row-major -> tiled
+    (direction 0) or back (direction 1); same shape and size.  The tiled kernels take both codes and parameters tiled."""
+    out = torch.empty_like(scales)
+    _check(lib().pot_repack_scales(_ptr(scales), _ptr(out), scales.shape[0], K, group, direction, _stream(stream)),
+           "pot_repack_scales")
+    return out
+
+
+def pot_layout_scale_index(N: int, K: int, group: int, row: int, g: int) -> int:
+    idx = ctypes.c_int64(-1)
+    _check(lib().pot_layout_scale_index(N, K, group, row, g, ctypes.byref(idx)), "pot_layout_scale_index")
+    return idx.value
 
 
 def uint_repack(packed: torch.Tensor, K: int, bits: int, direction: int = 0, stream=None) -> torch.Tensor:
@@ -263,31 +275,6 @@ def pot_gemv_noalloc(packed_tiled, scales, K: int, bits: int, group: int, x: tor
     _check(lib().pot_gemv_noalloc(_ptr(packed_tiled), _ptr(scales), packed_tiled.shape[0], K, bits, group, _ptr(x),
                                   _ptr(y), _stream(stream)), "pot_gemv_noalloc")
     return y
-
-
-class _GemvOp(ctypes.Structure):
-    _fields_ = [("packed_tiled", ctypes.c_void_p), ("scales_f16", ctypes.c_void_p), ("N", ctypes.c_int64),
-                ("K", ctypes.c_int64), ("group", ctypes.c_int), ("x_f16", ctypes.c_void_p), ("y_f16", ctypes.c_void_p),
-                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
-
-
-def pot_gemv_chain_prepare(ops, bits: int, stream=None) -> torch.Tensor:
-    """ops: sequence of (packed_tiled, scales, K, group, x, y, workspace-or-None) in execution order.  Returns the
-    device scratch that pot_gemv_chain_run takes (keep it, and the tensors of `ops`, alive while it is used)."""
-    n = len(ops)
-    arr = (_GemvOp * n)()
-    dev = ops[0][0].device
-    for i, (packed, scales, K, group, x, y, ws) in enumerate(ops):
-        arr[i] = _GemvOp(_ptr(packed), _ptr(scales), packed.shape[0], K, group, _ptr(x), _ptr(y), _ptr(ws),
-                         0 if ws is None else ws.numel())
-    scratch = torch.empty(int(lib().pot_gemv_chain_scratch_bytes(n)), dtype=torch.uint8, device=dev)
-    _check(lib().pot_gemv_chain_prepare(ctypes.cast(arr, ctypes.c_void_p), n, bits, _ptr(scratch), scratch.numel(),
-                                        _stream(stream)), "pot_gemv_chain_prepare")
-    return scratch
-
-
-def pot_gemv_chain_run(scratch: torch.Tensor, n_ops: int, bits: int, stream=None) -> None:
-    _check(lib().pot_gemv_chain_run(_ptr(scratch), n_ops, bits, _stream(stream)), "pot_gemv_chain_run")
 
 
 def pot_debug_errors() -> tuple[int, int, int]:

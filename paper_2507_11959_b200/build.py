@@ -38,6 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     OBJ_DIR.mkdir(exist_ok=True)
     nvcc = _nvcc()
     flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags += os.environ.get("POT_NVCC_FLAGS", "").split()  # extra compiler flags (experiments)
     if verbose:
         flags += ["-Xptxas", "-v"]
 

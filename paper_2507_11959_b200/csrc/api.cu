@@ -1,8 +1,40 @@
 // Host-only entry points: status strings, size helpers, the launch counter.
 #include "common.cuh"
 #include "layout.cuh"
+#include "sync.cuh"
 
 using namespace pot;
+
+// ---- device error words: one per kernel family, one definition for the whole library --------------------
+// In host code the array's name is only a handle for the runtime; its device address is looked up per GPU.
+static __device__ int g_error_words[3];
+
+namespace pot {
+int* error_ptr(int which) {
+    static std::atomic<int*> cache[64];
+    int dev = 0;
+    if (which < 0 || which > 2 || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    int* p = cache[dev].load(std::memory_order_acquire);
+    if (!p) {
+        void* q = nullptr;
+        if (cudaGetSymbolAddress(&q, g_error_words) != cudaSuccess) return nullptr;
+        p = (int*)q;
+        cache[dev].store(p, std::memory_order_release);
+    }
+    return p + which;
+}
+int error_fetch(int which) {
+    int v = -1, zero = 0;
+    if (which < 0 || which > 2) return -1;
+    if (cudaMemcpyFromSymbol(&v, g_error_words, sizeof(int), which * sizeof(int)) != cudaSuccess) return -1;
+    cudaMemcpyToSymbol(g_error_words, &zero, sizeof(int), which * sizeof(int));
+    return v;
+}
+}  // namespace pot
+
+extern "C" int pot_debug_gemv_error(void) { return error_fetch(ERR_GEMV); }
+extern "C" int pot_debug_gemm_error(void) { return error_fetch(ERR_GEMM); }
+extern "C" int pot_debug_prefill_error(void) { return error_fetch(ERR_PREFILL); }
 
 extern "C" const char* pot_status_string(pot_status_t s) {
     switch (s) {

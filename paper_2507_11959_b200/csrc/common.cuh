@@ -46,6 +46,8 @@ inline bool allow_max_dynamic_smem(K kernel) {
     cudaFuncAttributes fa;
     if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return false;
     const int room = kMaxDynamicSmem - (int)fa.sharedSizeBytes;  // static shared memory counts against the same limit
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        return false;
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, room) == cudaSuccess;
 }
 

@@ -13,7 +13,7 @@
 //  * otherwise, tiled layout: the tcgen05 kernel in gemm_prefill.cu.
 #include "common.cuh"
 #include "layout.cuh"
-#include "ring.cuh"
+#include "stream.cuh"
 
 namespace pot {
 
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
 #pragma unroll
             for (int i = 0; i < 2; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) rg_mma(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
+                for (int j = 0; j < 4; ++j) sk_mma(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
         }
     }
 #pragma unroll
@@ -130,11 +130,9 @@ static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout) {
     return M <= kSmallBatchAlways || gemm_prefill_wave_fill(M, N, K) < kMinWaveFill;
 }
 
-static int small_mt(int64_t) { return 1; }
-
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || M <= 0) return 0;
-    if (use_small(M, N, K, POT_LAYOUT_TILED)) return plan_ring(N, K, M, bits, 8 * small_mt(M)).ws_bytes;
+    if (use_small(M, N, K, POT_LAYOUT_TILED)) return plan_stream(N, K, M, bits, group, SK_POT, 8, 16).ws_bytes;
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
@@ -154,10 +152,10 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
         const size_t need = pot_gemm_workspace_bytes(M, N, K, bits, group);
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
         const int Mi = (int)M;
-#define POT_GS(B, T) return launch_ring<B, RG_POT_MMA, T>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, ring_error_ptr(), s)
-#define POT_GS_B(B) POT_GS(B, 1);
-        if (bits == 2) { POT_GS_B(2) } else if (bits == 3) { POT_GS_B(3) } else { POT_GS_B(4) }
-#undef POT_GS_B
+#define POT_GS(B) return launch_stream<B, SK_POT, 8, 16>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, error_ptr(ERR_GEMM), s)
+        if (bits == 2) POT_GS(2);
+        if (bits == 3) POT_GS(3);
+        POT_GS(4);
 #undef POT_GS
     }
     if (layout == POT_LAYOUT_TILED) {
@@ -175,4 +173,3 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
 // Diagnostic: reads and clears the device error word of the gemm kernels in this library (0 = every bounded
 // wait completed; 1 = a producer gave up waiting for a free ring slot; 2 = a consumer gave up waiting for
 // data).  Synchronises the device.
-extern "C" int pot_debug_gemm_error(void) { return ring_error_fetch(); }

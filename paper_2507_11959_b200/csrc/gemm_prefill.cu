@@ -23,7 +23,7 @@
 // Batches of up to 64 tokens run a variant with one tile of M token rows (the TMA box holds exactly M rows, the MMA's
 // N is M rounded up to 16), eight 24 KB stages and two TMA threads.
 //
-// All mbarrier waits are bounded (see ring.cuh); a wait that gives up records a code and the CTA carries
+// All mbarrier waits are bounded (see sync.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
 #include <cuda.h>
 
@@ -31,7 +31,7 @@
 
 #include "common.cuh"
 #include "layout.cuh"
-#include "ring.cuh"
+#include "sync.cuh"
 
 namespace pot {
 
@@ -289,7 +289,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
                     rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
                 }
-                const int64_t so = n * gpr + (cb0 + (kb >> 1)) * spg + (spg == 2 ? half : 0);
+                // tiled scales: the unit's values sit together, rows r and r + 8 of a group in one word
+                const int64_t so = (rb * ncb + cb0 + (kb >> 1)) * (16 * spg) + potl::scale_tile_index(r, spg == 2 ? half : 0);
                 sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
@@ -534,11 +535,10 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
     return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2>, 4, 2);
 }
 
-static int* prefill_error_ptr() { return ring_error_ptr(); }
+static int* prefill_error_ptr() { return error_ptr(ERR_PREFILL); }
 
 }  // namespace pot
 
 // Diagnostic: reads and clears the device error word of the prefill kernel (0 = every bounded wait completed;
 // 0x10 / 0x20 / 0x30 / 0x40 in the low byte = the TMA warp / the MMA warp / a dequant warp / the epilogue gave
 // up waiting, bits 8.. = the K block).  Synchronises the device.
-extern "C" int pot_debug_prefill_error(void) { return pot::ring_error_fetch(); }

@@ -1,23 +1,19 @@
-#include <vector>
-// Batch-1 decode GEMV, y = W~ x, fused with the dequantization (weights never touch HBM as
-// FP16).  CUDA-core kernels: codes are decoded in registers by the integer-add trick of
-// Sec. 4.2, products are accumulated in FP32 with the mixed-precision FMA
-// (fma.rn.f32.f16: FP16 operands, FP32 accumulator), K is reduced across lanes with warp
-// shuffles and, when N alone cannot fill 148 SMs, split across CTAs.
+#include <cstdlib>
+// Batch-1 decode GEMV, y = W~ x, fused with the dequantization (the weights never touch HBM as FP16).
 //
-//  * tiled layout (the fast path): the ring-buffered streaming kernel of ring.cuh.  One warp-step covers
-//    16 rows x 512 columns; a lane owns the 128-code records of two rows in one column block,
-//    i.e. exactly one quantization group per record (two for G = 64), so the scale pattern added
-//    to every pair is a loop constant.  The 16-byte loads of a warp cover whole 128-byte lines.
-//  * canonical layout (any N): one warp per row, 8 codes per lane per step.
+//  * tiled layout (the fast path): the streaming kernel of stream.cuh.  Every warp streams its own contiguous
+//    range of 16-row x 128-column units through a private shared-memory ring (bulk copies), decodes the codes in
+//    registers with the mask / shift / integer-add of Sec. 4.2 and feeds them, as A fragments, to warp-level
+//    tensor-core MMAs whose B columns all hold x; row blocks that span warps are combined in a fixed order.
+//  * canonical layout (any N): a CUDA-core kernel, one warp per row, 8 codes per lane per step, products
+//    accumulated in FP32 with the mixed-precision FMA and reduced across lanes with warp shuffles.
 //
-// Programmatic dependent launch: weights and scales do not depend on the previous kernel in
-// the stream, x does.  The kernels therefore issue their weight loads first and execute
-// griddepcontrol.wait only before the first read of x (and before any global write), so the
-// ramp-up of one GEMV overlaps the tail of the previous one.
+// Programmatic dependent launch: weights and scales do not depend on the previous kernel in the stream, x does.
+// The kernels request their first weights before they execute griddepcontrol.wait, and touch x, y and the
+// workspace only after it.
 #include "common.cuh"
 #include "layout.cuh"
-#include "ring.cuh"
+#include "stream.cuh"
 
 namespace pot {
 
@@ -82,24 +78,80 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
     if (lane == 0) y[row] = __float2half_rn(acc);
 }
 
+// Consumer warps per CTA of the streaming GEMV: 8 (two CTAs per SM: the next launch in the stream becomes resident and
+// fills its rings while this one computes) or 16 (one CTA per SM).
+static int gemv_warps() {
+    static const int w = [] {
+        const char* e = getenv("POT_GEMV_WARPS");
+        const int v = e ? atoi(e) : 16;
+        return (v == 8 || v == 24) ? v : 16;
+    }();
+    return w;
+}
+
+template <int KIND>
+static pot_status_t launch_gemv_stream(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
+                                       int bits, int group, const void* x, void* y, void* workspace, cudaStream_t s) {
+    int* err = error_ptr(ERR_GEMV);
+#define POT_SG(B, W) return launch_stream<B, KIND, 1, W>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s)
+    if (gemv_warps() == 8) {
+        if (bits == 2) POT_SG(2, 8);
+        if (bits == 3) POT_SG(3, 8);
+        POT_SG(4, 8);
+    }
+    if (gemv_warps() == 24) {
+        if (bits == 2) POT_SG(2, 24);
+        if (bits == 3) POT_SG(3, 24);
+        POT_SG(4, 24);
+    }
+    if (bits == 2) POT_SG(2, 16);
+    if (bits == 3) POT_SG(3, 16);
+    POT_SG(4, 16);
+#undef POT_SG
+}
+
+static size_t gemv_stream_workspace(int64_t N, int64_t K, int bits, int group, int tok) {
+    size_t need = 0;
+    for (int w : {8, 16, 24}) {
+        const StreamPlan p = plan_stream(N, K, 1, bits, group, SK_UINT, tok, w);
+        if (!p.ok) return 0;
+        if (p.ws_bytes > need) need = p.ws_bytes;
+    }
+    return need;
+}
+
 }  // namespace pot
 
 using namespace pot;
 
 extern "C" size_t pot_gemv_workspace_bytes(int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || N % 16 != 0) return 0;
-    return plan_ring(N, K, 1, bits, 1).ws_bytes;  // row-block step counters + FP32 partial slots
+    return gemv_stream_workspace(N, K, bits, group, 1);  // row-block arrival counters + FP32 partial slots
 }
 
-extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
-                                 pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes,
-                                 void* stream) {
+// every argument check of pot_gemv, run before anything is enqueued (also by the wrappers that enqueue copies first)
+static pot_status_t check_gemv_args(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                    pot_layout_t layout, const void* x, const void* y, const void* workspace, size_t ws_bytes) {
     if (!packed || !scales || !x || !y) return POT_ERR_NULL;
     pot_status_t st = check_shape(N, K, bits, group);
     if (st != POT_OK) return st;
     if (layout != POT_LAYOUT_CANONICAL && layout != POT_LAYOUT_TILED) return POT_ERR_UNSUPPORTED;
     if (!aligned16(packed) || !aligned16(scales) || !aligned16(x) || !aligned16(y) || !aligned16(workspace))
         return POT_ERR_ALIGN;
+    if (layout == POT_LAYOUT_TILED) {
+        if (N % 16 != 0) return POT_ERR_SHAPE;
+        if (!plan_stream(N, K, 1, bits, group, SK_POT, 1, 16).ok) return POT_ERR_SHAPE;
+        const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
+        if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
+    }
+    return POT_OK;
+}
+
+extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                 pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes,
+                                 void* stream) {
+    const pot_status_t st = check_gemv_args(packed, scales, N, K, bits, group, layout, x, y, workspace, ws_bytes);
+    if (st != POT_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
     if (layout == POT_LAYOUT_CANONICAL) {
         const dim3 grid((unsigned)((N + 7) / 8)), block(256);
@@ -109,19 +161,14 @@ extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t
         if (bits == 3) return launch_pdl(gemv_canonical_kernel<3, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
         return launch_pdl(gemv_canonical_kernel<4, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
     }
-    if (N % 16 != 0) return POT_ERR_SHAPE;
-    const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
-    if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
-    if (bits == 2) return launch_gemv_mma<2>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    if (bits == 3) return launch_gemv_mma<3>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    return launch_gemv_mma<4>(packed, scales, nullptr, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    return launch_gemv_stream<SK_POT>(packed, scales, nullptr, N, K, bits, group, x, y, workspace, s);
 }
 
 extern "C" pot_status_t pot_gemv_host(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
                                       pot_layout_t layout, const void* x_host, void* y_host, void* d_x, void* d_y,
                                       void* workspace, size_t ws_bytes, void* stream) {
-    if (!x_host || !y_host || !d_x || !d_y) return POT_ERR_NULL;
-    pot_status_t st = check_shape(N, K, bits, group);
+    if (!x_host || !y_host) return POT_ERR_NULL;
+    pot_status_t st = check_gemv_args(packed, scales, N, K, bits, group, layout, d_x, d_y, workspace, ws_bytes);
     if (st != POT_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemcpyAsync(d_x, x_host, (size_t)K * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return POT_ERR_CUDA;
@@ -155,9 +202,7 @@ extern "C" pot_status_t uint_gemv(const void* packed, const void* scales, const 
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);
     if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
     // same kernel as pot_gemv (tensor-core path); only the decode differs
-    if (bits == 2) return launch_gemv_mma<2, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    if (bits == 3) return launch_gemv_mma<3, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
-    return launch_gemv_mma<4, true>(packed, scales, zeros, N, K, group, x, y, workspace, ring_error_ptr(), s);
+    return launch_gemv_stream<SK_UINT>(packed, scales, zeros, N, K, bits, group, x, y, workspace, s);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -204,83 +249,12 @@ extern "C" pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* s
         g_noalloc_ptr[dev].store(p, std::memory_order_release);
         scratch = p;
     }
+    st = check_gemv_args(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, kNoAllocScratchBytes);
+    if (st != POT_OK) return st;  // nothing has been enqueued yet
     if (need == 0) return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, nullptr, 0, stream);
     // The array keeps whatever the previous call left in it.  Only the arrival counters have to start
     // at zero (the partial sums are fully overwritten before they are read), so clear just those.
-    const size_t counters_bytes = plan_ring(N, K, 1, bits, 1).ws_counters;
+    const size_t counters_bytes = plan_stream(N, K, 1, bits, group, SK_POT, 1, 16).ws_counters;
     if (cudaMemsetAsync(scratch, 0, counters_bytes, (cudaStream_t)stream) != cudaSuccess) return POT_ERR_CUDA;
     return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, need, stream);
 }
-
-// ---- chain of dependent GEMVs in one persistent kernel --------------------------------------------------
-constexpr size_t kChainHeader = 256;            // sync words of the kernel, then the operations
-constexpr size_t kChainSmem = 200 * 1024;       // every plan fits (plan_ring budgets 200 KB)
-
-extern "C" size_t pot_gemv_chain_scratch_bytes(int n_ops) {
-    return n_ops > 0 ? kChainHeader + (size_t)n_ops * sizeof(RingArgs) : 0;
-}
-
-extern "C" pot_status_t pot_gemv_chain_prepare(const pot_gemv_op_t* ops, int n_ops, int bits, void* scratch,
-                                               size_t scratch_bytes, void* stream) {
-    if (!ops || !scratch) return POT_ERR_NULL;
-    if (n_ops <= 0 || n_ops > (1 << 20)) return POT_ERR_SHAPE;
-    if (scratch_bytes < pot_gemv_chain_scratch_bytes(n_ops)) return POT_ERR_WORKSPACE;
-    if (!aligned16(scratch)) return POT_ERR_ALIGN;
-    std::vector<RingArgs> args((size_t)n_ops);
-    for (int i = 0; i < n_ops; ++i) {
-        const pot_gemv_op_t& o = ops[i];
-        if (!o.packed_tiled || !o.scales_f16 || !o.x_f16 || !o.y_f16) return POT_ERR_NULL;
-        const pot_status_t st = check_shape(o.N, o.K, bits, o.group);
-        if (st != POT_OK) return st;
-        if (o.N % 16 != 0) return POT_ERR_SHAPE;
-        if (!aligned16(o.packed_tiled) || !aligned16(o.scales_f16) || !aligned16(o.x_f16) || !aligned16(o.y_f16) ||
-            !aligned16(o.workspace))
-            return POT_ERR_ALIGN;
-        const RingPlan p = plan_ring(o.N, o.K, 1, bits, 1, rg_groups(RG_POT_MMA1));
-        if (!p.x_in_smem) return POT_ERR_UNSUPPORTED;
-        if (p.smem_bytes > kChainSmem) return POT_ERR_UNSUPPORTED;
-        if (p.ws_bytes > 0 && (!o.workspace || o.workspace_bytes < p.ws_bytes)) return POT_ERR_WORKSPACE;
-        args[(size_t)i] = ring_args(p, o.packed_tiled, o.scales_f16, nullptr, o.N, o.K, o.group, o.x_f16, 1, o.y_f16, o.workspace);
-    }
-    cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemsetAsync(scratch, 0, kChainHeader, s) != cudaSuccess) return POT_ERR_CUDA;
-    // pageable source: the runtime has consumed `args` when the call returns
-    if (cudaMemcpyAsync((char*)scratch + kChainHeader, args.data(), args.size() * sizeof(RingArgs), cudaMemcpyHostToDevice, s) !=
-        cudaSuccess)
-        return POT_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return POT_ERR_CUDA;
-    return POT_OK;
-}
-
-extern "C" pot_status_t pot_gemv_chain_run(const void* scratch, int n_ops, int bits, void* stream) {
-    if (!scratch) return POT_ERR_NULL;
-    if (n_ops <= 0) return POT_ERR_SHAPE;
-    if (bits < 2 || bits > 4) return POT_ERR_UNSUPPORTED;
-    unsigned* sync = (unsigned*)scratch;
-    const RingArgs* ops = (const RingArgs*)((const char*)scratch + kChainHeader);
-    int* err = ring_error_ptr();
-    auto run = [&](auto kernel) -> pot_status_t {
-        if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kSmCount);
-        cfg.blockDim = dim3(rg_threads(RG_POT_MMA1));
-        cfg.dynamicSmemBytes = kChainSmem;
-        cfg.stream = (cudaStream_t)stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeCooperative;  // the CTAs wait for one another: all must be resident
-        attr[0].val.cooperative = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, ops, n_ops, sync, err);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        return e == cudaSuccess ? POT_OK : POT_ERR_CUDA;
-    };
-    if (bits == 2) return run(ring_chain_kernel<2>);
-    if (bits == 3) return run(ring_chain_kernel<3>);
-    return run(ring_chain_kernel<4>);
-}
-
-// Diagnostic: reads and clears the device error word of the gemv kernels in this library (0 = every bounded
-// wait completed; 1 = a producer gave up waiting for a free ring slot; 2 = a consumer gave up waiting for
-// data).  Synchronises the device.
-extern "C" int pot_debug_gemv_error(void) { return ring_error_fetch(); }

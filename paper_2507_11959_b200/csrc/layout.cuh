@@ -94,14 +94,33 @@ __host__ __device__ inline BitPos record_bit(int bits, int kind, int q, int b) {
     return r;
 }
 
+// Tiled per-group parameters (scales, and the uniform twin's zero-points): the 16 * (128 / G) values of one unit
+// (16 rows x 128 columns) are stored together, units in the same [row block][column block] order as the codes, so a
+// kernel that streams a contiguous range of units streams a contiguous range of their scales too.  Inside a unit,
+// rows r and r + 8 of one group share a 32-bit word (r in the low half): halfword index ((s * 8 + r % 8) * 2 + r / 8)
+// for group s (0 .. 128/G - 1) of row r -- exactly the two rows a lane of the warp-level MMA owns.
+__host__ __device__ inline int scale_tile_index(int r, int s) { return (((s << 3) | (r & 7)) << 1) | (r >> 3); }
+// halfword index of the value of (row i, group g) in the tiled array
+__host__ __device__ inline int64_t scale_tiled_index(int64_t i, int64_t g, int64_t K, int G) {
+    const int spg = 128 / G;
+    const int64_t ncb = K / 128, cb = g / spg;
+    return ((i >> 4) * ncb + cb) * (16 * spg) + scale_tile_index((int)(i & 15), (int)(g - cb * spg));
+}
+
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------------------
 // Register decoders for the PoT byte-lane map.
 // rotated_words<BITS>(w, d): the quarter's n words -> its eight decoded words, every code rotated
 // into place (exponent from bit 2, sign at bit 7 of its byte lane) but NOT yet masked; decoded
-// word 7 of n = 3 is the exception: its bits sit two positions low (flagged by LOW7).
+// words whose bits wrap nowhere when shifted left are left unrotated, low(i) positions below their place.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t mad(uint32_t t, uint32_t c, uint32_t s) { return t * c + s; }
+// t * c + s as ONE multiply-add instruction (written in PTX: left to itself the compiler turns the power-of-two
+// multiplier into separate shift / logic / add instructions, which costs a third more issue slots in the decode)
+__device__ __forceinline__ uint32_t mad(uint32_t t, uint32_t c, uint32_t s) {
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(t), "r"(c), "r"(s));
+    return d;
+}
 __device__ __forceinline__ uint32_t rotr(uint32_t v, int s) { return __funnelshift_r(v, v, s); }
 __device__ __forceinline__ uint32_t rotl(uint32_t v, int s) { return __funnelshift_l(v, v, s); }
 // bitwise select: mask bits from a, the others from b (one LOP3)
@@ -112,11 +131,11 @@ struct PotLanes;
 template <>
 struct PotLanes<2> {
     static constexpr uint32_t MASK = 0x84848484u;
-    static constexpr bool LOW7 = false;
+    static __host__ __device__ constexpr int low(int i) { return (i & 3) == 0 ? 2 : 0; }
     static __device__ __forceinline__ void rotate(const uint32_t (&w)[2], uint32_t (&d)[8]) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            d[4 * k + 0] = rotl(w[k], 2);
+            d[4 * k + 0] = w[k];          // two positions low
             d[4 * k + 1] = w[k];
             d[4 * k + 2] = rotr(w[k], 2);
             d[4 * k + 3] = rotr(w[k], 4);
@@ -126,9 +145,9 @@ struct PotLanes<2> {
 template <>
 struct PotLanes<3> {
     static constexpr uint32_t MASK = 0x8C8C8C8Cu;
-    static constexpr bool LOW7 = true;
+    static __host__ __device__ constexpr int low(int i) { return i == 0 ? 1 : (i == 7 ? 2 : 0); }
     static __device__ __forceinline__ void rotate(const uint32_t (&w)[3], uint32_t (&d)[8]) {
-        d[0] = rotl(w[0], 1);
+        d[0] = w[0];                      // one position low
         d[1] = rotr(w[0], 1);
         d[2] = rotr(w[1], 2);
         d[3] = rotr(w[1], 4);
@@ -141,7 +160,7 @@ struct PotLanes<3> {
 template <>
 struct PotLanes<4> {
     static constexpr uint32_t MASK = 0x9C9C9C9Cu;
-    static constexpr bool LOW7 = false;
+    static __host__ __device__ constexpr int low(int) { return 0; }
     static __device__ __forceinline__ void rotate(const uint32_t (&w)[4], uint32_t (&d)[8]) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -165,13 +184,9 @@ __device__ __forceinline__ void pot_decode32(const uint32_t* rec, int T, uint32_
     L::rotate(w, d);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        if (L::LOW7 && i == 7) {
-            out[2 * i] = mad(d[i] & (MA >> 2), 1u << 10, sc2);
-            out[2 * i + 1] = mad(d[i] & (MB >> 2), 1u << 2, sc2);
-        } else {
-            out[2 * i] = mad(d[i] & MA, 1u << 8, sc2);
-            out[2 * i + 1] = (d[i] & MB) + sc2;
-        }
+        // fields that sit low(i) positions below their place: the alignment shift goes into the multiplier
+        out[2 * i] = mad(d[i] & (MA >> L::low(i)), 1u << (8 + L::low(i)), sc2);
+        out[2 * i + 1] = mad(d[i] & (MB >> L::low(i)), 1u << L::low(i), sc2);
     }
 }
 

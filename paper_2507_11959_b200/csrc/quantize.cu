@@ -171,9 +171,43 @@ __global__ void repack_backward_kernel(const uint32_t* __restrict__ src, uint32_
     }
 }
 
+// per-group parameters: row-major [N, K/G] <-> tiled (see scale_tiled_index); one thread per value
+__global__ void repack_scales_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int64_t N, int64_t K,
+                                     int G, int direction) {
+    const int64_t gpr = K / G, total = N * gpr;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t ti = potl::scale_tiled_index(t / gpr, t % gpr, K, G);
+        if (direction == 0) dst[ti] = src[t];
+        else dst[t] = src[ti];
+    }
+}
+
 }  // namespace pot
 
 using namespace pot;
+
+extern "C" pot_status_t pot_repack_scales(const void* src, void* dst, int64_t N, int64_t K, int group, int direction,
+                                          void* stream) {
+    if (!src || !dst) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, 2, group);
+    if (st != POT_OK) return st;
+    if (N % 16 != 0) return POT_ERR_SHAPE;
+    if (direction != 0 && direction != 1) return POT_ERR_UNSUPPORTED;
+    if (!aligned16(src) || !aligned16(dst)) return POT_ERR_ALIGN;
+    const int64_t total = N * (K / group);
+    const unsigned grid = (unsigned)((total + 255) / 256 < 65535 ? (total + 255) / 256 : 65535);
+    repack_scales_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const uint16_t*)src, (uint16_t*)dst, N, K, group, direction);
+    return launched();
+}
+
+extern "C" pot_status_t pot_layout_scale_index(int64_t N, int64_t K, int group, int64_t row, int64_t g, int64_t* index) {
+    if (!index) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, 2, group);
+    if (st != POT_OK) return st;
+    if (N % 16 != 0 || row < 0 || row >= N || g < 0 || g >= K / group) return POT_ERR_SHAPE;
+    *index = potl::scale_tiled_index(row, g, K, group);
+    return POT_OK;
+}
 
 extern "C" pot_status_t pot_quantize_ref(const void* W, int64_t N, int64_t K, int bits, int group,
                                          pot_scale_rule_t rule, void* scales, void* packed, void* stream) {

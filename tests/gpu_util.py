@@ -43,6 +43,11 @@ class PotCase:
         from paper_2507_11959_b200 import binding
         return binding.pot_repack(self.d_packed, self.K, self.bits, 0)
 
+    def tiled_S(self):
+        """scales in the tiled order that goes with tiled()"""
+        from paper_2507_11959_b200 import binding
+        return binding.pot_repack_scales(self.d_S, self.K, self.G, 0)
+
 
 class UintCase:
     def __init__(self, N, K, bits, G, dist="normal", sigma=0.02, seed=(0, 0), W_bits=None):
@@ -57,6 +62,14 @@ class UintCase:
     def tiled(self):
         from paper_2507_11959_b200 import binding
         return binding.uint_repack(self.d_packed, self.K, self.bits, 0)
+
+    def tiled_S(self):
+        from paper_2507_11959_b200 import binding
+        return binding.pot_repack_scales(self.d_S, self.K, self.G, 0)
+
+    def tiled_Z(self):
+        from paper_2507_11959_b200 import binding
+        return binding.pot_repack_scales(self.d_Z, self.K, self.G, 0)
 
 
 def gate(y_gpu_bits: np.ndarray, Y: np.ndarray, A: np.ndarray):

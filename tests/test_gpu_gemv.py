@@ -35,7 +35,7 @@ def test_pot_gemv_matches_oracle(B, oracle, bits, G):
         ok, worst, tight = gate(bits_of(y), Y[0], A[0])
         assert ok and tight < 4.0, ("canonical", N, K, worst, tight)
         if N % 16 == 0:
-            y = B.pot_gemv(c.tiled(), c.d_S, K, bits, G, f16_dev(X[0]), B.TILED)
+            y = B.pot_gemv(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X[0]), B.TILED)
             ok, worst, tight = gate(bits_of(y), Y[0], A[0])
             assert ok and tight < 4.0, ("tiled", N, K, worst, tight)
 
@@ -47,14 +47,14 @@ def test_pot_gemv_one_hot_returns_dequantized_column(B, oracle, bits):
     G, N, K = 64, 64, 1152
     c = PotCase(N, K, bits, G, dist="normal", seed=(4, 50 + bits))
     deq, _ = oracle.dequant(c.packed, c.S, K, bits, G)
-    tiled = c.tiled()
+    tiled, tiled_S = c.tiled(), c.tiled_S()
     for j in (0, 1, 2, 3, 63, 64, 127, 128, 129, 500, 511, 512, 1023, 1151):
         x = np.zeros(K, dtype=np.uint16)
         x[j] = 0x3C00
-        for layout, P in ((B.CANONICAL, c.d_packed), (B.TILED, tiled)):
-            y = bits_of(B.pot_gemv(P, c.d_S, K, bits, G, f16_dev(x), layout))
+        for layout, P, S in ((B.CANONICAL, c.d_packed, c.d_S), (B.TILED, tiled, tiled_S)):
+            y = bits_of(B.pot_gemv(P, S, K, bits, G, f16_dev(x), layout))
             assert np.array_equal(y, deq[:, j]), (layout, j)
-            Yg = bits_of(B.pot_gemm(P, c.d_S, K, bits, G, f16_dev(x).reshape(1, K), layout))
+            Yg = bits_of(B.pot_gemm(P, S, K, bits, G, f16_dev(x).reshape(1, K), layout))
             assert np.array_equal(Yg[0], deq[:, j]), ("gemm", layout, j)
 
 
@@ -63,17 +63,17 @@ def test_pot_gemv_closed_form_and_determinism(B, oracle):
     assert B.pot_gemv_workspace_bytes(N, K, bits, G) > 0
     c = PotCase(N, K, bits, G, dist="t5", seed=(4, 60))
     x = f16_dev(acts(1, K, 160)[0])
-    tiled = c.tiled()
+    tiled, tiled_S = c.tiled(), c.tiled_S()
     ws = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, bits, G))
-    y0 = bits_of(B.pot_gemv(tiled, c.d_S, K, bits, G, x, B.TILED, workspace=ws))
+    y0 = bits_of(B.pot_gemv(tiled, tiled_S, K, bits, G, x, B.TILED, workspace=ws))
     for _ in range(5):  # same workspace reused: counters must come back to zero; sums in fixed order
-        assert np.array_equal(bits_of(B.pot_gemv(tiled, c.d_S, K, bits, G, x, B.TILED, workspace=ws)), y0)
+        assert np.array_equal(bits_of(B.pot_gemv(tiled, tiled_S, K, bits, G, x, B.TILED, workspace=ws)), y0)
     # all codes 0 (sign +, E = 0), x = 1: y_i = G * sum_g S_ig
     S = np.full((16, 4), 0x2000, dtype=np.uint16)
     S[:, 1] = 0x2400
     packed = np.zeros((16, 512 * bits // 8), dtype=np.uint8)
     ones = f16_dev(np.full(512, 0x3C00, dtype=np.uint16))
-    y = B.pot_gemv(B.pot_repack(to_dev(packed), 512, bits, 0), f16_dev(S), 512, bits, 128, ones, B.TILED)
+    y = B.pot_gemv(B.pot_repack(to_dev(packed), 512, bits, 0), B.pot_repack_scales(f16_dev(S), 512, 128, 0), 512, bits, 128, ones, B.TILED)
     assert torch.all(y.float() == 128 * (3 * 2.0 ** -7 + 2.0 ** -6))
 
 
@@ -88,7 +88,7 @@ def test_uint_gemv_matches_oracle(B, oracle, bits, G):
         ok, worst, tight = gate(bits_of(y), Y[0], A[0])
         assert ok and tight < 4.0, ("canonical", N, K, worst, tight)
         if N % 16 == 0:
-            y = B.uint_gemv(c.tiled(), c.d_S, c.d_Z, K, bits, G, f16_dev(X[0]), B.TILED)
+            y = B.uint_gemv(c.tiled(), c.tiled_S(), c.tiled_Z(), K, bits, G, f16_dev(X[0]), B.TILED)
             ok, worst, tight = gate(bits_of(y), Y[0], A[0])
             assert ok and tight < 4.0, ("tiled", N, K, worst, tight)
 
@@ -101,11 +101,11 @@ def test_pot_gemm_small_batch_matches_oracle(B, oracle, bits, M):
         c = PotCase(N, K, bits, G, dist="t5", seed=(4, 500 + 10 * bits + i))
         X = acts(M, K, 600 + i)
         Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
-        Yg = B.pot_gemm(c.tiled(), c.d_S, K, bits, G, f16_dev(X), B.TILED)
+        Yg = B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X), B.TILED)
         ok, worst, tight = gate(bits_of(Yg), Y, A)
         assert ok and tight < 4.0, ("small", N, K, M, worst, tight)
         # every row of the batch equals the separate GEMV within the gate
-        y0 = B.pot_gemv(c.tiled(), c.d_S, K, bits, G, f16_dev(X[M - 1]), B.TILED)
+        y0 = B.pot_gemv(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X[M - 1]), B.TILED)
         assert gate(bits_of(y0), Y[M - 1], A[M - 1])[0]
 
 
@@ -129,12 +129,12 @@ def test_gemv_with_activations_too_long_for_shared_memory(B, oracle):
     X = acts(1, K, 900)
     c = PotCase(N, K, bits, G, dist="t5", seed=(4, 900))
     Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
-    y = B.pot_gemv(c.tiled(), c.d_S, K, bits, G, f16_dev(X[0]), B.TILED)
+    y = B.pot_gemv(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X[0]), B.TILED)
     ok, worst, tight = gate(bits_of(y), Y[0], A[0])
     assert ok and tight < 4.0, ("pot", worst, tight)
     u = UintCase(N, K, bits, G, dist="t5", seed=(4, 901))
     Y, A = oracle.uint_matmul(u.packed, u.S, u.Z, K, bits, G, X)
-    y = B.uint_gemv(u.tiled(), u.d_S, u.d_Z, K, bits, G, f16_dev(X[0]), B.TILED)
+    y = B.uint_gemv(u.tiled(), u.tiled_S(), u.tiled_Z(), K, bits, G, f16_dev(X[0]), B.TILED)
     ok, worst, tight = gate(bits_of(y), Y[0], A[0])
     assert ok and tight < 4.0, ("uint", worst, tight)
     assert B.pot_debug_errors() == (0, 0, 0)

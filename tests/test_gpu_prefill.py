@@ -30,7 +30,7 @@ def test_prefill_gemm_matches_oracle(B, oracle, bits, G):
         c = PotCase(N, K, bits, G, dist="normal", sigma=0.015, seed=(5, 10 * bits + i))
         X = synth.activations(synth.rng_for(5, 100 + i), M, K, outliers=(i % 2 == 1))
         Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
-        Yg = B.pot_gemm(c.tiled(), c.d_S, K, bits, G, f16_dev(X), B.TILED)
+        Yg = B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X), B.TILED)
         assert B.pot_debug_errors() == (0, 0, 0)
         ok, worst, tight = gate(bits_of(Yg), Y, A)
         assert ok and tight < 4.0, (M, N, K, worst, tight)
@@ -47,8 +47,8 @@ def test_split_k_workspace_is_reusable(B, oracle):
     assert need > 0
     ws = B.new_workspace(need)
     dX = f16_dev(X)
-    y1 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
-    y2 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
+    y1 = bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, dX, B.TILED, workspace=ws))
+    y2 = bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, dX, B.TILED, workspace=ws))
     assert B.pot_debug_errors() == (0, 0, 0)
     assert np.array_equal(y1, y2)
     ok, worst, tight = gate(y1, Y, A)
@@ -62,9 +62,9 @@ def test_two_issuers_give_the_same_bits_every_time(B, oracle):
     c = PotCase(N, K, bits, G, dist="t5", seed=(5, 88))
     dX = f16_dev(synth.activations(synth.rng_for(5, 188), M, K, outliers=True))
     ws = B.new_workspace(B.pot_gemm_workspace_bytes(M, N, K, bits, G))
-    y0 = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws))
+    y0 = bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, dX, B.TILED, workspace=ws))
     for _ in range(4):
-        assert np.array_equal(bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, dX, B.TILED, workspace=ws)), y0)
+        assert np.array_equal(bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, dX, B.TILED, workspace=ws)), y0)
     assert B.pot_debug_errors() == (0, 0, 0)
 
 
@@ -77,7 +77,7 @@ def test_prefill_one_hot_tokens_return_dequantized_columns(B, oracle, bits):
     ks = (np.arange(M) * 37 + 5) % K
     X = np.zeros((M, K), dtype=np.uint16)
     X[np.arange(M), ks] = 0x3C00
-    Yg = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, f16_dev(X), B.TILED))
+    Yg = bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X), B.TILED))
     assert np.array_equal(Yg, deq[:, ks].T)
 
 
@@ -86,7 +86,7 @@ def test_prefill_config5_shape_sampled(B, oracle):
     bits, G, M, N, K = 3, 128, 2048, 10240, 8192
     c = PotCase(N, K, bits, G, dist="normal", sigma=0.015, seed=(5, 70))
     X = synth.activations(synth.rng_for(5, 71), M, K, outliers=False)
-    Yg = bits_of(B.pot_gemm(c.tiled(), c.d_S, K, bits, G, f16_dev(X), B.TILED))
+    Yg = bits_of(B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X), B.TILED))
     assert B.pot_debug_errors() == (0, 0, 0)
     rows = np.unique(np.concatenate([[0, 1, 127, 128, 255, N - 129, N - 128, N - 1],
                                      synth.rng_for(5, 72).integers(0, N, 24)])).astype(np.int64)

@@ -17,14 +17,14 @@ def test_noalloc_gemv_matches_workspace_gemv_twice_in_a_row(oracle):
     need = B.pot_gemv_workspace_bytes(N, K, bits, G)
     assert 0 < need <= B.pot_gemv_noalloc_max_scratch_bytes()
     c = PotCase(N, K, bits, G, dist="t5", seed=(6, 1))
-    tiled = c.tiled()
+    tiled, tiled_S = c.tiled(), c.tiled_S()
     Y, A = None, None
     for call in range(2):  # second call finds the first call's leftovers in the shared array
         X = synth.activations(synth.rng_for(6, 10 + call), 1, K)
         x = f16_dev(X[0])
-        ref = B.pot_gemv(tiled, c.d_S, K, bits, G, x, B.TILED)            # existing entry, caller workspace
+        ref = B.pot_gemv(tiled, tiled_S, K, bits, G, x, B.TILED)            # existing entry, caller workspace
         y = torch.empty(N, dtype=torch.float16, device="cuda")
-        B.pot_gemv_noalloc(tiled, c.d_S, K, bits, G, x, y)                 # new entry, built-in scratch
+        B.pot_gemv_noalloc(tiled, tiled_S, K, bits, G, x, y)                 # new entry, built-in scratch
         torch.cuda.synchronize()
         assert np.array_equal(bits_of(y), bits_of(ref)), f"call {call}"   # same kernel, same summation order
         Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
@@ -34,7 +34,7 @@ def test_noalloc_gemv_matches_workspace_gemv_twice_in_a_row(oracle):
 
 def test_noalloc_gemv_rejects_shapes_beyond_its_scratch():
     from paper_2507_11959_b200 import binding as B
-    bits, G, N, K = 3, 128, 65536, 11008
+    bits, G, N, K = 3, 128, 262144, 11008
     assert B.pot_gemv_workspace_bytes(N, K, bits, G) > B.pot_gemv_noalloc_max_scratch_bytes()
     a = torch.zeros(16, dtype=torch.uint8, device="cuda")   # never read: the size check comes first
     fake_packed = torch.empty((N, 16), dtype=torch.uint8, device="cuda")  # only its row count is used
