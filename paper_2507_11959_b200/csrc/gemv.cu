@@ -1,4 +1,3 @@
-#include <cstdlib>
 // Batch-1 decode GEMV, y = W~ x, fused with the dequantization (the weights never touch HBM as FP16).
 //
 //  * tiled layout (the fast path): the streaming kernel of stream.cuh.  Every warp streams its own contiguous
@@ -78,42 +77,38 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
     if (lane == 0) y[row] = __float2half_rn(acc);
 }
 
-// Consumer warps per CTA of the streaming GEMV: 8 (two CTAs per SM: the next launch in the stream becomes resident and
-// fills its rings while this one computes) or 16 (one CTA per SM).
-static int gemv_warps() {
-    static const int w = [] {
-        const char* e = getenv("POT_GEMV_WARPS");
-        const int v = e ? atoi(e) : 16;
-        return (v == 8 || v == 24) ? v : 16;
-    }();
-    return w;
+// CTAs per SM of the streaming GEMV (16 consumer warps each).  Two: the next launch in the stream becomes resident,
+// sets itself up and fills its rings while this one computes, which hides the launch and the prologue (about 2.5 us);
+// the price is 64 registers per thread and half the ring, i.e. a slower loop (about 15 %).  Worth it while a CTA's
+// share of the matrix is small; one CTA per SM otherwise, and whenever the half-size ring could not hold two slots.
+constexpr size_t kTwoCtaMaxShare = 300 * 1024;  // bytes of codes + scales per CTA
+static int gemv_occupancy(int64_t N, int64_t K, int bits, int group, int kind) {
+    const StreamPlan p2 = plan_stream(N, K, 1, bits, group, kind, 1, 16, 2);
+    if (!p2.ok || !p2.x_in_smem || p2.stages < 2 || p2.grid < kSmCount) return 1;
+    const size_t share = (size_t)(N / 16) * (size_t)(K / 128) * (size_t)(sk_slot_bytes(bits, group, kind) / SK_Q) / (size_t)p2.grid;
+    return share <= kTwoCtaMaxShare ? 2 : 1;
 }
 
 template <int KIND>
 static pot_status_t launch_gemv_stream(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
                                        int bits, int group, const void* x, void* y, void* workspace, cudaStream_t s) {
     int* err = error_ptr(ERR_GEMV);
-#define POT_SG(B, W) return launch_stream<B, KIND, 1, W>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s)
-    if (gemv_warps() == 8) {
-        if (bits == 2) POT_SG(2, 8);
-        if (bits == 3) POT_SG(3, 8);
-        POT_SG(4, 8);
+#define POT_SG(B, O) return launch_stream<B, KIND, 1, 16, O>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s)
+    if (gemv_occupancy(N, K, bits, group, KIND) == 2) {
+        if (bits == 2) POT_SG(2, 2);
+        if (bits == 3) POT_SG(3, 2);
+        POT_SG(4, 2);
     }
-    if (gemv_warps() == 24) {
-        if (bits == 2) POT_SG(2, 24);
-        if (bits == 3) POT_SG(3, 24);
-        POT_SG(4, 24);
-    }
-    if (bits == 2) POT_SG(2, 16);
-    if (bits == 3) POT_SG(3, 16);
-    POT_SG(4, 16);
+    if (bits == 2) POT_SG(2, 1);
+    if (bits == 3) POT_SG(3, 1);
+    POT_SG(4, 1);
 #undef POT_SG
 }
 
 static size_t gemv_stream_workspace(int64_t N, int64_t K, int bits, int group, int tok) {
     size_t need = 0;
-    for (int w : {8, 16, 24}) {
-        const StreamPlan p = plan_stream(N, K, 1, bits, group, SK_UINT, tok, w);
+    for (int occ : {1, 2}) {  // the partial-sum layout does not depend on the occupancy, the check is for safety
+        const StreamPlan p = plan_stream(N, K, 1, bits, group, SK_UINT, tok, 16, occ);
         if (!p.ok) return 0;
         if (p.ws_bytes > need) need = p.ws_bytes;
     }
@@ -258,3 +253,7 @@ extern "C" pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* s
     if (cudaMemsetAsync(scratch, 0, counters_bytes, (cudaStream_t)stream) != cudaSuccess) return POT_ERR_CUDA;
     return pot_gemv(packed_tiled, scales, N, K, bits, group, POT_LAYOUT_TILED, x, y, scratch, need, stream);
 }
+
+#ifdef SK_TRACE
+extern "C" void pot_debug_set_trace(void* p) { pot::g_sk_trace = (unsigned long long*)p; }
+#endif

@@ -54,10 +54,12 @@ struct StreamPlan {
     size_t x_bytes, smem_bytes;
     int max_slots;        // partial-sum slots per row block
     size_t ws_counters, ws_bytes;
+    bool aligned;         // CTA ranges end on row-block boundaries (no partial sums cross CTAs)
+    int nrb;
     bool ok;              // false: the shape cannot run on this kernel (too many units)
 };
 
-inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int group, int kind, int tok, int warps) {
+inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int group, int kind, int tok, int warps, int occ = 1) {
     StreamPlan p = {};
     const int64_t nrb = N / 16, ncb = K / 128, U = nrb * ncb;
     p.ok = U > 0 && U < (int64_t(1) << 31) && ncb < (1 << 24);
@@ -72,9 +74,14 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     p.grid = (int)(grid < kSmCount ? grid : kSmCount);
     p.gw_total = (uint32_t)((int64_t)p.grid * warps < U ? (int64_t)p.grid * warps : U);
     const int64_t GW = (int64_t)p.gw_total;
-    const int64_t per_warp = (U + GW - 1) / GW;
-    // shared memory: header, the staged activations, W rings.  W = 8: two CTAs share an SM.
-    const size_t budget = (warps <= 8 ? 112 : 224) * 1024;
+    // Row-block split: no sums cross CTAs, at the price of CTAs that differ by one row block.  Taken when that costs at
+    // most a fifth more than the even split and every warp of a CTA still gets a unit.
+    p.nrb = (int)nrb;
+    const int64_t rb_min = nrb / p.grid, rb_max = (nrb + p.grid - 1) / p.grid;
+    p.aligned = nrb >= p.grid && p.grid == kSmCount && rb_min * ncb >= warps && (double)rb_max * p.grid <= 1.2 * (double)nrb;
+    const int64_t per_warp = p.aligned ? (rb_max * ncb + warps - 1) / warps : (U + GW - 1) / GW;
+    // shared memory: header, the staged activations, W rings
+    const size_t budget = (occ == 2 ? 113 : 224) * 1024;  // two CTAs per SM: 228 KB less 1 KB reserve each
     const size_t hdr = (size_t)sk_header_bytes(warps, tok);
     const size_t slot = (size_t)sk_slot_bytes(bits, group, kind);
     const size_t xb = (size_t)(tok > 1 ? 8 : 1) * (size_t)K * 2;
@@ -109,6 +116,10 @@ struct StreamArgs {
     uint32_t units, gw_total;      // U, grid * W
     int ncb, group, stages, x_bytes, max_slots, M;
     int fits32;                    // U * gw_total < 2^32: 32-bit range arithmetic
+    int aligned, nrb;              // row-block split (see the kernel), number of row blocks
+#ifdef SK_TRACE
+    unsigned long long* trace;     // [launch slot][cta][8] globaltimer stamps
+#endif
 };
 
 #ifdef __CUDACC__
@@ -129,10 +140,10 @@ __device__ __forceinline__ uint32_t sk_muldiv(uint32_t a, uint32_t b, uint32_t c
 
 // KIND: SK_POT / SK_UINT.  TOK = 1: GEMV (x in every B column).  TOK = 8: up to 8 tokens, one per B column.
 // XSMEM: the activations are staged in shared memory in fragment order (else they are read through L1 from global).
-// W consumer warps per CTA; W = 8 leaves room for a second CTA on the SM, so that the next launch in the stream can
-// become resident and fill its rings while this one still computes.
-template <int BITS, int KIND, int TOK, bool XSMEM, int W>
-__global__ void __launch_bounds__(W * 32, W <= 8 ? 2 : 1)
+// W consumer warps per CTA; OCC = 2 leaves room for a second CTA on the SM (64 registers per thread, half the shared
+// memory), so that the next launch in the stream can become resident and fill its rings while this one still computes.
+template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1>
+__global__ void __launch_bounds__(W * 32, OCC)
 stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     constexpr int UB = sk_unit_bytes(BITS);
     constexpr bool UNIFORM = (KIND == SK_UINT);
@@ -140,6 +151,18 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;  // MMA fragment coordinates: rows gid and gid + 8, quarter tig
+#ifdef SK_TRACE
+    auto stamp = [&](int i) {
+        if (sa.trace && lane == 0 && (warp == 0 || warp == W - 1)) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            sa.trace[((size_t)blockIdx.x * 2 + (warp ? 1 : 0)) * 8 + i] = t;
+        }
+    };
+    stamp(0);
+#else
+    auto stamp = [&](int) {};
+#endif
     const int S = sa.stages;
     const int spg = 128 / sa.group;
     const uint32_t PB = 32u * (uint32_t)spg;                 // parameter bytes of one unit
@@ -154,10 +177,19 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     const uint32_t ring = smem0 + (uint32_t)HDR + (uint32_t)sa.x_bytes + (uint32_t)warp * (uint32_t)S * slot_bytes;
 
     // ---- this warp's range of units [a, b) ---------------------------------------------------------------
-    const uint32_t U = sa.units, GW = sa.gw_total;
-    const uint32_t gw = blockIdx.x * W + warp;
+    // Unit split (sa.aligned == 0): the U units are cut into GW equal ranges, warp gw = blockIdx * W + warp takes range gw.
+    // Row-block split (sa.aligned == 1): CTA c takes the row blocks [c nrb / grid, (c + 1) nrb / grid) and its W warps
+    // cut that range of units into W equal ranges -- no row block is shared between CTAs.
     const bool f32 = sa.fits32 != 0;
-    const uint32_t a = gw < GW ? sk_muldiv(gw, U, GW, f32) : 0u, b = gw < GW ? sk_muldiv(gw + 1, U, GW, f32) : 0u;
+    uint32_t base = 0, U = sa.units, GW = sa.gw_total, gw = blockIdx.x * W + warp;
+    if (sa.aligned) {
+        const uint32_t r0 = sk_muldiv(blockIdx.x, (uint32_t)sa.nrb, gridDim.x, f32), r1 = sk_muldiv(blockIdx.x + 1, (uint32_t)sa.nrb, gridDim.x, f32);
+        base = r0 * (uint32_t)sa.ncb;
+        U = (r1 - r0) * (uint32_t)sa.ncb;
+        GW = W;
+        gw = (uint32_t)warp;
+    }
+    const uint32_t a = base + (gw < GW ? sk_muldiv(gw, U, GW, f32) : 0u), b = base + (gw < GW ? sk_muldiv(gw + 1, U, GW, f32) : 0u);
     const uint32_t n = b - a;
     const uint32_t nchunks = (n + SK_Q - 1) / SK_Q;
 
@@ -174,12 +206,13 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         bulk_g2s(dst + SK_Q * UB, ps + (size_t)j * SK_Q * PB, cnt * PB, bar);
         if constexpr (UNIFORM) bulk_g2s(dst + SK_Q * (UB + PB), pz + (size_t)j * SK_Q * PB, cnt * PB, bar);
     };
-    if (lane == 0) {
-        for (int s = 0; s < S; ++s) mbar_init(bars + (uint32_t)s * 8u, 1);
+    if (lane < S) {  // lane s sets up slot s and requests chunk s: the weights do not depend on the predecessor
+        mbar_init(bars + (uint32_t)lane * 8u, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (uint32_t j = 0; j < (uint32_t)S && j < nchunks; ++j) issue(j, j);  // weights do not depend on the predecessor
+        if ((uint32_t)lane < nchunks) issue((uint32_t)lane, (uint32_t)lane);
     }
     __syncwarp();
+    stamp(7);
     pdl_launch_dependents();
 
     // ---- row blocks of the range; which of its segments are partial, and their place among the contributors
@@ -187,7 +220,10 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     uint32_t rb = a / ncb, cb = a - rb * ncb;
     const uint32_t rb0 = rb, rbL = n ? (b - 1) / ncb : rb;
     uint32_t slot0 = 0, exp0 = 0, expL = 0;  // exp == 0: the segment covers its whole row block
-    auto owner = [&](uint32_t u) { return f32 ? ((u + 1) * GW - 1) / U : (uint32_t)((((uint64_t)u + 1) * GW - 1) / U); };
+    auto owner = [&](uint32_t u) {  // the warp (numbered like gw) whose range holds unit u
+        u -= base;
+        return f32 ? ((u + 1) * GW - 1) / U : (uint32_t)((((uint64_t)u + 1) * GW - 1) / U);
+    };
     if (n) {
         if (cb != 0 || b < (rb0 + 1) * ncb) {
             const uint32_t lo = owner(rb0 * ncb), hi = owner((rb0 + 1) * ncb - 1);
@@ -197,12 +233,14 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         if (rbL != rb0 && b != (rbL + 1) * ncb) expL = owner((rbL + 1) * ncb - 1) - gw + 1;  // this warp is its first contributor
     }
     // a row block whose contributors all sit in this CTA is combined in shared memory
-    const uint32_t cta_lo = blockIdx.x * W;
+    const uint32_t cta_lo = sa.aligned ? 0u : blockIdx.x * W;
     const bool loc0 = exp0 && gw - slot0 >= cta_lo && gw - slot0 + exp0 <= cta_lo + W;
     const bool locL = expL && gw + expL <= cta_lo + W;
     if (threadIdx.x < W) lcnt[threadIdx.x] = 0u;
 
+    stamp(1);
     pdl_wait();  // x, Y and the workspace may belong to the previous kernel in the stream
+    stamp(2);
     if constexpr (XSMEM) {
         uint4* dst = reinterpret_cast<uint4*>(smem + HDR);
         const uint4* src = reinterpret_cast<const uint4*>(sa.X);
@@ -219,6 +257,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         }
     }
     __syncthreads();
+    stamp(3);
 
     float acc[2][4];
 #pragma unroll
@@ -387,6 +426,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         if (!mbar_test(bar, phase) && !mbar_wait(bar, phase)) {
             if (err && lane == 0) atomicCAS(err, 0, 2 | (int)(j << 8) | (warp << 24));
         }
+        if (j == 0) stamp(4);
         if (left >= (uint32_t)SK_Q && cb + (uint32_t)SK_Q <= ncb) {
             // the common case: a full chunk inside one row block, straight-line code
 #pragma unroll
@@ -419,10 +459,15 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             phase ^= 1u;
         }
     }
+    stamp(5);
     if (n && cb != 0) deliver(rb);
+    stamp(6);
 }
 #endif  // __CUDACC__
 
+#ifdef SK_TRACE
+inline unsigned long long* g_sk_trace = nullptr;   // next launch's trace block (advanced per launch)
+#endif
 // ---- host side --------------------------------------------------------------------------------------------
 inline StreamArgs stream_args(const StreamPlan& p, const void* packed, const void* scales, const void* zeros, int64_t N,
                               int64_t K, int group, const void* X, int M, void* Y, void* workspace) {
@@ -438,29 +483,35 @@ inline StreamArgs stream_args(const StreamPlan& p, const void* packed, const voi
     sa.K = K;
     sa.units = p.units;
     sa.gw_total = p.gw_total;
+    sa.aligned = p.aligned ? 1 : 0;
+    sa.nrb = p.nrb;
     sa.ncb = p.ncb;
     sa.group = group;
     sa.stages = p.stages;
     sa.x_bytes = (int)p.x_bytes;
     sa.max_slots = p.max_slots;
     sa.M = M;
+#ifdef SK_TRACE
+    sa.trace = g_sk_trace;
+    if (g_sk_trace) g_sk_trace += 148 * 2 * 8;
+#endif
     sa.fits32 = ((uint64_t)p.units + 1) * ((uint64_t)sa.gw_total + 1) < (uint64_t(1) << 32) ? 1 : 0;
     return sa;
 }
 
 #ifdef __CUDACC__
-template <int BITS, int KIND, int TOK, int W>
+template <int BITS, int KIND, int TOK, int W, int OCC = 1>
 pot_status_t launch_stream(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                            const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
-    const StreamPlan p = plan_stream(N, K, M, BITS, group, KIND, TOK, W);
+    const StreamPlan p = plan_stream(N, K, M, BITS, group, KIND, TOK, W, OCC);
     if (!p.ok) return POT_ERR_SHAPE;
     const StreamArgs sa = stream_args(p, packed, scales, zeros, N, K, group, X, M, Y, workspace);
     auto run = [&](auto kernel) -> pot_status_t {
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(W * 32), p.smem_bytes, s, sa, err);
     };
-    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W>);
-    return run(stream_kernel<BITS, KIND, TOK, false, W>);
+    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC>);
+    return run(stream_kernel<BITS, KIND, TOK, false, W, OCC>);
 }
 #endif
 
