@@ -24,7 +24,7 @@ EXPORTS = [
     "pot_status_string", "pot_packed_bytes", "pot_scales_bytes", "pot_gemv_workspace_bytes",
     "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack", "pot_repack_scales", "pot_layout_scale_index",
     "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_host", "pot_gemm", "uint_quantize_ref", "uint_dequant",
-    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemm_error", "pot_debug_prefill_error",
+    "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemv_plan", "pot_debug_gemm_error", "pot_debug_prefill_error",
 ]
 
 _lib = None
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.pot_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.uint_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.pot_repack_scales.argtypes = [vp, vp, i64, i64, i32, i32, vp]
+        L.pot_debug_gemv_plan.argtypes = [i64, i64, i32, i32, i32, vp, vp, vp, vp]
         L.pot_layout_scale_index.argtypes = [i64, i64, i32, i64, i64, vp]
         L.pot_dequant.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.pot_gemv.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
@@ -275,6 +276,13 @@ def pot_gemv_noalloc(packed_tiled, scales, K: int, bits: int, group: int, x: tor
     _check(lib().pot_gemv_noalloc(_ptr(packed_tiled), _ptr(scales), packed_tiled.shape[0], K, bits, group, _ptr(x),
                                   _ptr(y), _stream(stream)), "pot_gemv_noalloc")
     return y
+
+
+def pot_debug_gemv_plan(N: int, K: int, bits: int, group: int, uniform: bool = False) -> dict:
+    """{'ctas_per_sm', 'row_block_split', 'ring_slots', 'x_in_smem'} of the tiled GEMV launch for this shape."""
+    v = [ctypes.c_int(-1) for _ in range(4)]
+    _check(lib().pot_debug_gemv_plan(N, K, bits, group, 1 if uniform else 0, *[ctypes.byref(x) for x in v]), "pot_debug_gemv_plan")
+    return dict(zip(("ctas_per_sm", "row_block_split", "ring_slots", "x_in_smem"), (x.value for x in v)))
 
 
 def pot_debug_errors() -> tuple[int, int, int]:

@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
 constexpr size_t kTwoCtaMaxShare = 300 * 1024;  // bytes of codes + scales per CTA
 static int gemv_occupancy(int64_t N, int64_t K, int bits, int group, int kind) {
     const StreamPlan p2 = plan_stream(N, K, 1, bits, group, kind, 1, 16, 2);
-    if (!p2.ok || !p2.x_in_smem || p2.stages < 2 || p2.grid < kSmCount) return 1;
+    if (!p2.ok || !p2.x_in_smem || p2.ring_capacity < 2 || p2.grid < kSmCount) return 1;
     const size_t share = (size_t)(N / 16) * (size_t)(K / 128) * (size_t)(sk_slot_bytes(bits, group, kind) / SK_Q) / (size_t)p2.grid;
     return share <= kTwoCtaMaxShare ? 2 : 1;
 }
@@ -118,6 +118,24 @@ static size_t gemv_stream_workspace(int64_t N, int64_t K, int bits, int group, i
 }  // namespace pot
 
 using namespace pot;
+
+// Host arithmetic only: how pot_gemv / uint_gemv would run a tiled shape (tests assert which variants they reach).
+extern "C" pot_status_t pot_debug_gemv_plan(int64_t N, int64_t K, int bits, int group, int uniform, int* ctas_per_sm,
+                                            int* row_block_split, int* ring_slots, int* x_in_smem) {
+    if (!ctas_per_sm || !row_block_split || !ring_slots || !x_in_smem) return POT_ERR_NULL;
+    pot_status_t st = check_shape(N, K, bits, group);
+    if (st != POT_OK) return st;
+    if (N % 16 != 0) return POT_ERR_SHAPE;
+    const int kind = uniform ? SK_UINT : SK_POT;
+    const int occ = gemv_occupancy(N, K, bits, group, kind);
+    const StreamPlan p = plan_stream(N, K, 1, bits, group, kind, 1, 16, occ);
+    if (!p.ok) return POT_ERR_SHAPE;
+    *ctas_per_sm = occ;
+    *row_block_split = p.aligned ? 1 : 0;
+    *ring_slots = p.stages;
+    *x_in_smem = p.x_in_smem ? 1 : 0;
+    return POT_OK;
+}
 
 extern "C" size_t pot_gemv_workspace_bytes(int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || N % 16 != 0) return 0;

@@ -47,26 +47,51 @@ __global__ void __launch_bounds__(256) quantize_kernel(const __half* __restrict_
             sb = __half_as_ushort(S[gi]);
         } else if (rule == POT_SCALE_SEARCH) {
             // Algorithm 1: s0 = max|w| / (2^q_max - 1); b = 0.01 i, i = 1..200; keep the first minimiser of
-            // Q1(b) = sum (w - s0 b sign(w) 2^E(b))^2.  The per-lane partial sums are combined in a fixed
-            // butterfly order, so the choice is deterministic.
+            // Q1(b) = sum_k (w_k - s0 b sign(w_k) 2^E_k(b))^2.  The 200 candidates are spread over the lanes
+            // (lane l takes i = l + 1, l + 33, ...), every lane adds the G terms of its candidates in the order
+            // k = 0 .. G-1 with separately rounded multiply and add -- the order and rounding of a plain sequential
+            // loop -- and the warp takes the smallest (Q1, i) pair.  The weights travel by shuffle.
             const double s0 = amax / (double)((1 << QMAX) - 1);
+            constexpr int NC = 7;  // ceil(200 / 32)
+            double sc[NC], q1[NC];
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                sc[c] = __dmul_rn(s0, __dmul_rn(0.01, (double)(lane + 1 + 32 * c)));
+                q1[c] = 0.0;
+            }
+            for (int src = 0; src < 32; ++src) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (j < per) {
+                        const double wk = __shfl_sync(0xffffffffu, w[j], src);
+                        const double w2 = __dmul_rn(wk, wk);
+#pragma unroll
+                        for (int c = 0; c < NC; ++c) {
+                            const double s2 = __dmul_rn(sc[c], sc[c]);
+                            int E = 0;
+#pragma unroll
+                            for (int k = 0; k < QMAX; ++k) E += (w2 > __dmul_rn(s2, (double)(1 << (2 * k + 1)))) ? 1 : 0;
+                            double rec = __dmul_rn(sc[c], (double)(1 << E));
+                            if (wk < 0.0) rec = -rec;
+                            const double d = (sc[c] > 0.0) ? __dsub_rn(wk, rec) : wk;
+                            q1[c] = __dadd_rn(q1[c], __dmul_rn(d, d));
+                        }
+                    }
+                }
+            }
             double qmin = 1e300;
             int best = 1;
-            for (int i = 1; i <= 200; ++i) {
-                const double sc = s0 * (0.01 * (double)i);
-                double q1 = 0.0;
-                for (int j = 0; j < per; ++j) {
-                    int E = 0;
-                    for (int k = 0; k < QMAX; ++k) E += (w[j] * w[j] > ldexp(sc * sc, 2 * k + 1)) ? 1 : 0;
-                    double rec = ldexp(sc, E);
-                    if (w[j] < 0.0) rec = -rec;
-                    const double d = (sc > 0.0) ? (w[j] - rec) : w[j];
-                    q1 += d * d;
-                }
-                for (int o = 16; o; o >>= 1) q1 += __shfl_xor_sync(0xffffffffu, q1, o);
-                if (q1 < qmin) { qmin = q1; best = i; }
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int i = lane + 1 + 32 * c;
+                if (i <= 200 && q1[c] < qmin) { qmin = q1[c]; best = i; }
             }
-            sb = clamp_scale_bits(__half_as_ushort(__double2half(s0 * (0.01 * (double)best))), BITS);
+            for (int o = 16; o; o >>= 1) {  // smallest Q1, ties to the smaller i
+                const double qo = __shfl_xor_sync(0xffffffffu, qmin, o);
+                const int bo = __shfl_xor_sync(0xffffffffu, best, o);
+                if (qo < qmin || (qo == qmin && bo < best)) { qmin = qo; best = bo; }
+            }
+            sb = clamp_scale_bits(__half_as_ushort(__double2half(__dmul_rn(s0, __dmul_rn(0.01, (double)best)))), BITS);
             if (lane == 0) S[gi] = __ushort_as_half(sb);
         } else {
             const double s = (rule == POT_SCALE_TOP) ? ldexp(amax, -QMAX) : amax / (double)((1 << QMAX) - 1);

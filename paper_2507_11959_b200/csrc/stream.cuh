@@ -49,6 +49,7 @@ struct StreamPlan {
     uint32_t units;       // U
     uint32_t gw_total;    // GW: warps that own a range (grid * W, or U when there are fewer units than that)
     int stages;           // S: slots per warp ring
+    int ring_capacity;    // slots per warp that would fit
     int tok;              // B columns in use: 1 (GEMV) or 8 (small batch)
     bool x_in_smem;
     size_t x_bytes, smem_bytes;
@@ -89,6 +90,7 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     p.x_in_smem = hdr + xb + ring2 <= budget;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
     int64_t st = (int64_t)((budget - hdr - p.x_bytes) / ((size_t)warps * slot));
+    p.ring_capacity = (int)(st > 8 ? 8 : st);
     const int64_t need = (per_warp + SK_Q - 1) / SK_Q;
     if (st > need) st = need;
     if (st > 8) st = 8;

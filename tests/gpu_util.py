@@ -81,3 +81,109 @@ def gate(y_gpu_bits: np.ndarray, Y: np.ndarray, A: np.ndarray):
     ok = err <= 1e-3 * A + 1e-5
     tight = err / (2.0 ** -10 * np.abs(Y) + 2.0 ** -20 * A + 1e-30)
     return bool(ok.all()), float((err / (1e-3 * A + 1e-5)).max()), float(tight.max())
+
+
+# ---- stray-write detection ------------------------------------------------------------------------------------
+# compute-sanitizer is not available to these tests, so every output and workspace of a parity test sits between two
+# pads of a seeded byte pattern that must still be intact after the call.
+_PAD = 4096
+_pattern = None
+
+
+def _pad_pattern() -> torch.Tensor:
+    global _pattern
+    if _pattern is None:
+        g = torch.Generator().manual_seed(2507119590)
+        _pattern = torch.randint(0, 256, (_PAD,), dtype=torch.uint8, generator=g).to(DEV)
+    return _pattern
+
+
+class Guarded:
+    """A device buffer of `shape` / `dtype` with a 4 KB canary pad on both sides."""
+
+    def __init__(self, shape, dtype, zero: bool = False):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.n = (n + 15) // 16 * 16
+        self.buf = torch.empty(self.n + 2 * _PAD, dtype=torch.uint8, device=DEV)
+        self.buf[:_PAD] = _pad_pattern()
+        self.buf[_PAD + self.n:] = _pad_pattern()
+        self.view = self.buf[_PAD:_PAD + n].view(dtype).reshape(shape)
+        if zero:
+            self.buf[_PAD:_PAD + self.n] = 0
+
+    def intact(self) -> bool:
+        return bool(torch.equal(self.buf[:_PAD], _pad_pattern()) and torch.equal(self.buf[_PAD + self.n:], _pad_pattern()))
+
+
+class GuardedBinding:
+    """The binding with every output and workspace it allocates placed between canary pads; after each call the
+    device is synchronised and the pads are checked.  Anything else is forwarded unchanged."""
+
+    def __init__(self):
+        from paper_2507_11959_b200 import binding
+        binding.lib()
+        self._b = binding
+
+    def __getattr__(self, name):
+        return getattr(self._b, name)
+
+    def _finish(self, what, *guards):
+        torch.cuda.synchronize()
+        for g in guards:
+            assert g is None or g.intact(), f"{what}: a write landed outside its buffer"
+
+    def _ws(self, nbytes):
+        return Guarded((nbytes,), torch.uint8, zero=True) if nbytes else None
+
+    def pot_dequant(self, packed, scales, K, bits, group, out_dtype=0, **kw):
+        out = Guarded((packed.shape[0], K), torch.float16 if out_dtype == 0 else torch.bfloat16)
+        self._b.pot_dequant(packed, scales, K, bits, group, out_dtype, out=out.view, **kw)
+        self._finish("pot_dequant", out)
+        return out.view
+
+    def uint_dequant(self, packed, scales, zeros, K, bits, group, kernel=0, **kw):
+        out = Guarded((packed.shape[0], K), torch.float16)
+        self._b.uint_dequant(packed, scales, zeros, K, bits, group, kernel, out=out.view, **kw)
+        self._finish("uint_dequant", out)
+        return out.view
+
+    def pot_gemv(self, packed, scales, K, bits, group, x, layout=0, workspace=None, **kw):
+        N = packed.shape[0]
+        y = Guarded((N,), torch.float16)
+        ws = None
+        if workspace is None and layout == self._b.TILED:
+            ws = self._ws(self._b.pot_gemv_workspace_bytes(N, K, bits, group))
+            workspace = None if ws is None else ws.view
+        self._b.pot_gemv(packed, scales, K, bits, group, x, layout, y=y.view, workspace=workspace, **kw)
+        self._finish("pot_gemv", y, ws)
+        return y.view
+
+    def uint_gemv(self, packed, scales, zeros, K, bits, group, x, layout=0, workspace=None, **kw):
+        N = packed.shape[0]
+        y = Guarded((N,), torch.float16)
+        ws = None
+        if workspace is None and layout == self._b.TILED:
+            ws = self._ws(self._b.pot_gemv_workspace_bytes(N, K, bits, group))
+            workspace = None if ws is None else ws.view
+        self._b.uint_gemv(packed, scales, zeros, K, bits, group, x, layout, y=y.view, workspace=workspace, **kw)
+        self._finish("uint_gemv", y, ws)
+        return y.view
+
+    def pot_gemm(self, packed, scales, K, bits, group, X, layout=0, workspace=None, **kw):
+        N, M = packed.shape[0], X.shape[0]
+        Y = Guarded((M, N), torch.float16)
+        ws = None
+        if workspace is None and layout == self._b.TILED:
+            ws = self._ws(self._b.pot_gemm_workspace_bytes(M, N, K, bits, group))
+            workspace = None if ws is None else ws.view
+        self._b.pot_gemm(packed, scales, K, bits, group, X, layout, Y=Y.view, workspace=workspace, **kw)
+        self._finish("pot_gemm", Y, ws)
+        return Y.view
+
+    def new_workspace(self, nbytes, device=DEV):
+        """A zeroed, guarded workspace; keep the returned tensor's guard alive through `guard_of`."""
+        if nbytes == 0:
+            return None
+        g = Guarded((nbytes,), torch.uint8, zero=True)
+        g.view._guard = g
+        return g.view

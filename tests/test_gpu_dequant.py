@@ -12,9 +12,8 @@ SHAPES = [(1, 128), (3, 384), (37, 1152), (256, 4096), (130, 2176)]  # several t
 
 @pytest.fixture(scope="module")
 def B():
-    from paper_2507_11959_b200 import binding
-    binding.lib()
-    return binding
+    from tests.gpu_util import GuardedBinding
+    return GuardedBinding()  # outputs and workspaces between canary pads, checked after every call
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -57,15 +56,14 @@ def test_validate_scales_counts_illegal_entries(B):
 @pytest.mark.parametrize("bits", [2, 3, 4])
 def test_scale_search_rule_matches_algorithm_1(B, oracle, bits):
     from paper_2507_11959_b200 import synth
-    G, N, K = 128, 48, 1024
-    W = synth.weights(synth.rng_for(3, 70 + bits), N, K, "normal")
+    G, N, K = 128, 96, 2048
+    W = synth.weights(synth.rng_for(3, 70 + bits), N, K, "normal" if bits != 3 else "t5")
     S_ref, bstar = oracle.scale_search(W, bits, G)
     packed, S = B.pot_quantize_ref(f16_dev(W), bits, G, B.SCALE_SEARCH)
     Sg = bits_of(S)
-    same = Sg == S_ref
-    # both sides decide in FP64; a different summation order may flip the argmin only between
-    # candidates whose objective values agree to rounding, which must stay very rare
-    assert same.mean() > 0.995
+    # both sides add the 128 squared errors of a candidate in the same order with the same FP64 roundings, so the
+    # argmin -- index work -- must agree for every group, not just for most
+    assert np.array_equal(Sg, S_ref), np.argwhere(Sg != S_ref)[:5]
     codes, _ = oracle.quantize(W, bits, G, oracle.RULE_GIVEN, Sg)
     assert np.array_equal(packed.cpu().numpy(), oracle.pack(codes, bits))
 

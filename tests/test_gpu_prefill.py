@@ -10,9 +10,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def B():
-    from paper_2507_11959_b200 import binding
-    binding.lib()
-    return binding
+    from tests.gpu_util import GuardedBinding
+    return GuardedBinding()  # outputs and workspaces between canary pads, checked after every call
 
 
 # (M, N, K).  M <= 64 runs the one-token-tile variant (eight stages, a TMA box of exactly M rows, two TMA threads), larger
