@@ -85,7 +85,7 @@ constexpr size_t kTwoCtaMaxShare = 300 * 1024;  // bytes of codes + scales per C
 static int gemv_occupancy(int64_t N, int64_t K, int bits, int group, int kind) {
     const StreamPlan p2 = plan_stream(N, K, 1, bits, group, kind, 1, 16, 2);
     if (!p2.ok || !p2.x_in_smem || p2.ring_capacity < 2 || p2.grid < kSmCount) return 1;
-    const size_t share = (size_t)(N / 16) * (size_t)(K / 128) * (size_t)(sk_slot_bytes(bits, group, kind) / SK_Q) / (size_t)p2.grid;
+    const size_t share = (size_t)(N / 16) * (size_t)(K / 128) * (size_t)sk_unit_total_bytes(bits, group, kind) / (size_t)p2.grid;
     return share <= kTwoCtaMaxShare ? 2 : 1;
 }
 

@@ -29,14 +29,15 @@ namespace pot {
 
 enum StreamKind { SK_POT = 0, SK_UINT = 1 };
 
-constexpr int SK_Q = 4;  // units per chunk (one ring slot, one set of bulk copies)
+constexpr int SK_QMAX = 4;  // units per chunk (one ring slot, one set of bulk copies): 4, or 2 where 4 would leave one slot
 
 __host__ __device__ constexpr int sk_unit_bytes(int bits) { return 256 * bits; }
 // bytes of one ring slot: Q units of codes, then their scales (then their zero-points)
 __host__ __device__ constexpr int sk_param_bytes(int group) { return 16 * (128 / group) * 2; }
-__host__ __device__ constexpr int sk_slot_bytes(int bits, int group, int kind) {
-    return SK_Q * (sk_unit_bytes(bits) + (kind == SK_UINT ? 2 : 1) * sk_param_bytes(group));
+__host__ __device__ constexpr int sk_unit_total_bytes(int bits, int group, int kind) {
+    return sk_unit_bytes(bits) + (kind == SK_UINT ? 2 : 1) * sk_param_bytes(group);
 }
+__host__ __device__ constexpr int sk_slot_bytes(int bits, int group, int kind, int q) { return q * sk_unit_total_bytes(bits, group, kind); }
 
 // shared-memory header of a CTA: W x 8 full barriers, W local arrival counters, W x 2 local partial-sum slots
 __host__ __device__ constexpr int sk_header_bytes(int warps, int tok) {
@@ -48,6 +49,7 @@ struct StreamPlan {
     int ncb;              // column blocks (units per row block)
     uint32_t units;       // U
     uint32_t gw_total;    // GW: warps that own a range (grid * W, or U when there are fewer units than that)
+    int q;                // Q: units per slot
     int stages;           // S: slots per warp ring
     int ring_capacity;    // slots per warp that would fit
     int tok;              // B columns in use: 1 (GEMV) or 8 (small batch)
@@ -84,14 +86,18 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     // shared memory: header, the staged activations, W rings
     const size_t budget = (occ == 2 ? 113 : 224) * 1024;  // two CTAs per SM: 228 KB less 1 KB reserve each
     const size_t hdr = (size_t)sk_header_bytes(warps, tok);
-    const size_t slot = (size_t)sk_slot_bytes(bits, group, kind);
     const size_t xb = (size_t)(tok > 1 ? 8 : 1) * (size_t)K * 2;
+    // slots of 4 units unless the ring could then hold only one of them next to the staged activations
+    int q = SK_QMAX;
+    if (hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget) q = 2;
+    p.q = q;
+    const size_t slot = (size_t)sk_slot_bytes(bits, group, kind, q);
     const size_t ring2 = (size_t)warps * 2 * slot;  // at least two slots per warp
     p.x_in_smem = hdr + xb + ring2 <= budget;
     p.x_bytes = p.x_in_smem ? (xb + 127) / 128 * 128 : 0;
     int64_t st = (int64_t)((budget - hdr - p.x_bytes) / ((size_t)warps * slot));
     p.ring_capacity = (int)(st > 8 ? 8 : st);
-    const int64_t need = (per_warp + SK_Q - 1) / SK_Q;
+    const int64_t need = (per_warp + q - 1) / q;
     if (st > need) st = need;
     if (st > 8) st = 8;
     if (st < 1) st = 1;
@@ -144,7 +150,7 @@ __device__ __forceinline__ uint32_t sk_muldiv(uint32_t a, uint32_t b, uint32_t c
 // XSMEM: the activations are staged in shared memory in fragment order (else they are read through L1 from global).
 // W consumer warps per CTA; OCC = 2 leaves room for a second CTA on the SM (64 registers per thread, half the shared
 // memory), so that the next launch in the stream can become resident and fill its rings while this one still computes.
-template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1>
+template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1, int SK_Q = SK_QMAX>
 __global__ void __launch_bounds__(W * 32, OCC)
 stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     constexpr int UB = sk_unit_bytes(BITS);
@@ -377,7 +383,6 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         }
         // the scale words {row gid, row gid + 8} of this lane's group
         const uint32_t poff = ((spg == 2 ? (uint32_t)(tig >> 1) * 8u : 0u) + (uint32_t)gid) * 4u;
-        const uint32_t scw = sk_lds32(param + poff);
         uint32_t lo[16], hi[16];
         if constexpr (!UNIFORM) {
             // plane k of a unit holds word k of every (row, quarter): this lane's word sits at byte 4 * lane
@@ -386,11 +391,13 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             for (int h = 0; h < 2; ++h)
 #pragma unroll
                 for (int k = 0; k < BITS; ++k) w[h][k] = sk_lds32(code + (uint32_t)(k * 256 + h * 128) + (uint32_t)lane * 4u);
+            const uint32_t scw = sk_lds32(param + poff);  // {row gid, row gid + 8}
             potl::pot_decode32<BITS, 1>(w[0], 0, __byte_perm(scw, 0, 0x1010), lo);
             potl::pot_decode32<BITS, 1>(w[1], 0, __byte_perm(scw, 0, 0x3232), hi);
         } else {
             // the quarter's words sit at record words 2 tig, 2 tig + 1 (n = 2), 2 tig, 2 tig + 1, 8 + tig (n = 3) or
             // 4 tig .. 4 tig + 3 (n = 4); record word w is byte (w / 4) * 256 + row * 16 + (w % 4) * 4
+            const uint32_t scw = sk_lds32(param + poff);
             const uint32_t zw = sk_lds32(param + SK_Q * PB + poff);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -512,8 +519,12 @@ pot_status_t launch_stream(const void* packed, const void* scales, const void* z
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(W * 32), p.smem_bytes, s, sa, err);
     };
-    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC>);
-    return run(stream_kernel<BITS, KIND, TOK, false, W, OCC>);
+    if (p.q == 2) {
+        if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2>);
+        return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2>);
+    }
+    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, SK_QMAX>);
+    return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, SK_QMAX>);
 }
 #endif
 
