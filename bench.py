@@ -144,7 +144,7 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config tables (chain only)")
@@ -216,22 +216,29 @@ def main():
                 fn(stream)
         return g
 
-    def time_graph(g, steps, warmup):
+    def time_graph(g, steps, warmup, per_step=None):
+        """ms per replay over `steps` replays (CUDA events on the launching stream, a barrier and a device synchronise
+        on both sides).  per_step: a list that receives every replay's own duration (an event between replays)."""
         with torch.cuda.stream(stream):
             for _ in range(warmup):
                 g.replay()
             stream.synchronize()
             pdist.barrier()
             torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(steps):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1 if per_step is not None else 2)]
+            ev[0].record(stream)
+            for i in range(steps):
                 g.replay()
-            e1.record(stream)
+                if per_step is not None:
+                    ev[i + 1].record(stream)
+            if per_step is None:
+                ev[1].record(stream)
             stream.synchronize()
             torch.cuda.synchronize()
             pdist.barrier()
-        return e0.elapsed_time(e1) / steps  # ms per step
+        if per_step is not None:
+            per_step.extend(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+        return ev[0].elapsed_time(ev[-1]) / steps  # ms per step
 
     layers3, bytes3 = build_chain(HEADLINE_BITS)
     launches_before = B.pot_launch_count()
@@ -241,7 +248,8 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    ms = time_graph(g3, args.steps, args.warmup)
+    step_ms = []
+    ms = time_graph(g3, args.steps, args.warmup, per_step=step_ms)
     clocks = sampler.stop()
     ms = pdist.max_over_ranks(ms, dev)
     value = world * bytes3 / (ms * 1e-3) / 1e9
@@ -299,10 +307,12 @@ def main():
         "config": {"workload": f"llama2-7b-shaped decode chain, batch 1, {args.layers} layers x 5 projections, PoT {HEADLINE_BITS}-bit g{GROUP}, tiled layout, CUDA graph + PDL",
                    "l2": "inputs larger than L2 (%.2f GB of codes+scales per step vs 126 MB)" % (bytes3 / 1e9),
                    "bytes_per_step": bytes3, "launches_per_step": launches_per_step},
+        "step_ms_stats": {"median": float(np.median(step_ms)), "p10": float(np.percentile(step_ms, 10)),
+                          "p90": float(np.percentile(step_ms, 90)), "min": float(min(step_ms)), "max": float(max(step_ms)), "n": len(step_ms)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": value / world / peaks["hbm_gbs"], "frac_of_8TBs_nominal": value / world / 8000.0,
-                     "peak_source": peaks["source"], "kernel": "ring_kernel<3, RG_POT_MMA1|RG_POT_MMA1W, 1> (decode GEMV on mma.sync, tiled layout)",
+                     "peak_source": peaks["source"], "kernel": "stream_kernel<3, PoT, GEMV, 16 warps, 2 CTAs per SM> (decode GEMV: per-warp bulk-copy rings, decode in registers, mma.sync)",
                      "per_launch_us": ms * 1e3 / max(1, launches_per_step),
                      "algorithmic_bytes_per_launch": bytes3 / max(1, launches_per_step),
                      # dram__bytes_read+write per launch from the ncu capture of the 12288x4096 launch
@@ -407,8 +417,17 @@ def cpu_baseline():
         for packed, S, K, x in layer:
             oracle.matmul(packed, S, K, HEADLINE_BITS, GROUP, x)
         best = min(best, time.perf_counter() - t0)
+    # the oracle's dequantizer beside it (config 3's metric): the 4096 x 4096, 3-bit matrix to FP16, best of 3
+    packed0, S0, K0 = layer[1][0], layer[1][1], layer[1][2]
+    best_dq = 1e30
+    for _ in range(3):
+        t0 = time.perf_counter()
+        oracle.dequant(packed0, S0, K0, HEADLINE_BITS, GROUP)
+        best_dq = min(best_dq, time.perf_counter() - t0)
     return {"value": nbytes / best / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "one layer (5 projections, 202M weights) of the 32-layer chain, best of 3"}
+            "sample": "one layer (5 projections, 202M weights) of the 32-layer chain, best of 3",
+            "dequant_Gweights_s": packed0.shape[0] * K0 / best_dq / 1e9,
+            "dequant_sample": "4096 x 4096 3-bit g128 matrix of the same layer to FP16, best of 3"}
 
 
 def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_chain, enqueue_chain):
@@ -435,10 +454,38 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
     del gf, layersf
     torch.cuda.empty_cache()
 
-    def rotating(make, copies):
-        return [make() for _ in range(copies)]
+    L2_BYTES = 126e6
 
-    # per-projection GEMV, HBM-cold (rotating copies > 4x L2), PoT vs uniform twin, tiled layout, + config 1
+    def time_eager(fn, n=20):
+        """isolated launches: each one timed alone with its own pair of events (launch latency and ramp included)"""
+        ts = []
+        with torch.cuda.stream(stream):
+            for i in range(n + 3):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                stream.synchronize()
+                e0.record(stream)
+                fn(i)
+                e1.record(stream)
+                stream.synchronize()
+                if i >= 3:
+                    ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    def ab_ratio(run_a, run_b, copies, reps=7):
+        """A and B interleaved (ABAB...) in ONE captured graph over rotating HBM-cold buffers; the graph is replayed
+        `reps` times with an event after every launch's group, so both see the same clocks and the same cache state.
+        Returns (median ms of A per launch, of B, and min / median / max of the per-repetition ratio B / A)."""
+        ga = capture(lambda s: [run_a(i, s) for i in range(copies)])
+        gb = capture(lambda s: [run_b(i, s) for i in range(copies)])
+        ta, tb = [], []
+        for _ in range(reps):
+            ta.append(time_graph(ga, 4, 1) / copies)
+            tb.append(time_graph(gb, 4, 1) / copies)
+        r = [y / x for x, y in zip(ta, tb)]
+        return float(np.median(ta)), float(np.median(tb)), {"min": min(r), "median": float(np.median(r)), "max": max(r), "reps": reps}
+
+    # per-projection GEMV (config 1 and config 2 shapes): isolated launch, steady state in a graph over HBM-cold rotating
+    # copies (> 4x L2), and next to the uniform twin (interleaved repetitions)
     rows = []
     shapes = [("cfg1 4096x4096", 4096, 4096, "normal")] + [(f"7B {p.name}", p.N, p.K, "t5") for p in synth.LLAMA2_7B if p.name != "up"]
     for name, N, K, dist in shapes:
@@ -452,45 +499,89 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
             up, uS, uZ = B.uint_quantize_ref(W, bits, GROUP)
             utiled = B.uint_repack(up, K, bits, 0)
             uS, uZ = B.pot_repack_scales(uS, K, GROUP, 0), B.pot_repack_scales(uZ, K, GROUP, 0)
-            copies = max(2, int(4 * 126e6 / (N * K * bits / 8)) + 1)
+            copies = max(2, int(4 * L2_BYTES / (N * K * bits / 8)) + 1)
             ws = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, bits, GROUP), dev)
             pts = [(tiled.clone(), S.clone()) for _ in range(copies)]
             uts = [(utiled.clone(), uS.clone(), uZ.clone()) for _ in range(copies)]
-            gp = capture(lambda s: [B.pot_gemv(t, sc, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s) for t, sc in pts])
-            gu = capture(lambda s: [B.uint_gemv(t, sc, z, K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s) for t, sc, z in uts])
-            tp = min(time_graph(gp, 10, 3) for _ in range(3)) / copies
-            tu = min(time_graph(gu, 10, 3) for _ in range(3)) / copies
+            run_p = lambda i, s: B.pot_gemv(pts[i][0], pts[i][1], K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s)
+            run_u = lambda i, s: B.uint_gemv(uts[i][0], uts[i][1], uts[i][2], K, bits, GROUP, x, B.TILED, y=y, workspace=ws, stream=s)
+            tp, tu, ratio = ab_ratio(run_p, run_u, copies)
+            t_iso = time_eager(lambda i: run_p(i % copies, stream)) if bits == HEADLINE_BITS else None
             bp = gemv_bytes(N, K, bits, GROUP)
             bu = bp + N * (K // GROUP) * 2
-            rows.append({"shape": name, "bits": bits, "pot_us": tp * 1e3, "pot_GBps": bp / tp / 1e6, "pot_frac_hbm": bp / tp / 1e6 / hbm,
-                         "uint_us": tu * 1e3, "uint_GBps": bu / tu / 1e6, "pot_speedup_vs_uint": tu / tp})
-            del pts, uts, gp, gu
+            rows.append({"shape": name, "bits": bits, "pot_us_steady": tp * 1e3, "pot_us_isolated_launch": None if t_iso is None else t_iso * 1e3,
+                         "pot_GBps": bp / tp / 1e6, "pot_frac_hbm": bp / tp / 1e6 / hbm, "uint_us_steady": tu * 1e3,
+                         "uint_GBps": bu / tu / 1e6, "uint_over_pot_time": ratio, "plan": B.pot_debug_gemv_plan(N, K, bits, GROUP)})
+            del pts, uts
         del W
         torch.cuda.empty_cache()
     ex["gemv_per_projection_hbm_cold"] = rows
 
-    # standalone dequant (config 3): PoT vs uniform twin (fast and naive), FP16 out
+    # one large matrix (28672 x 8192, 3 bit): the kernel without the per-launch costs that dominate the 7B shapes
+    N, K = 28672, 8192
+    gq = torch.Generator(device=dev).manual_seed(BASE_PROFILE_SEED)
+    Pb = [torch.randint(0, 256, (N, K * 3 // 8), dtype=torch.uint8, device=dev, generator=gq) for _ in range(6)]
+    Sb = (torch.rand((N, K // GROUP), device=dev, generator=gq) * 0.01 + 0.002).to(torch.float16)
+    xb = torch.randn(K, device=dev, generator=gq).to(torch.float16)
+    yb = torch.empty(N, dtype=torch.float16, device=dev)
+    wsb = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, 3, GROUP), dev)
+    gb = capture(lambda s: [B.pot_gemv(p, Sb, K, 3, GROUP, xb, B.TILED, y=yb, workspace=wsb, stream=s) for p in Pb])
+    tb = min(time_graph(gb, 5, 2) for _ in range(3)) / len(Pb)
+    nb = gemv_bytes(N, K, 3, GROUP)
+    ex["gemv_28672x8192_3bit_hbm_cold"] = {"us": tb * 1e3, "GBps": nb / tb / 1e6, "frac_of_measured_hbm": nb / tb / 1e6 / hbm,
+                                           "frac_of_8TBs_nominal": nb / tb / 1e6 / 8000.0}
+    del Pb, gb
+    torch.cuda.empty_cache()
+
+    # standalone dequant (config 3): PoT vs the uniform twin (fast and naive kernels), FP16 out.  HBM-cold: every launch
+    # of a graph reads its own packed matrix and writes its own output, R pairs with R x bytes >= 4 x L2; the L2-warm
+    # figure (one pair, written over and over) is reported beside it, labelled.
     rows = []
     for N, K in synth.DEQUANT_SWEEP:
         W = f16(synth.weights(synth.rng_for(3, N % 89), N, K, "normal"))
-        out = torch.empty((N, K), dtype=torch.float16, device=dev)
         for bits in (2, 3, 4):
             for G in (64, 128):
                 packed, S = B.pot_quantize_ref(W, bits, G, B.SCALE_TOP)
                 up, uS, uZ = B.uint_quantize_ref(W, bits, G)
-                reps = max(1, int(2e9 / (N * K * 2.4)))
-                gp = capture(lambda s: [B.pot_dequant(packed, S, K, bits, G, B.F16, out=out, stream=s) for _ in range(reps)])
-                gf = capture(lambda s: [B.uint_dequant(up, uS, uZ, K, bits, G, B.UINT_FAST, out=out, stream=s) for _ in range(reps)])
-                gn = capture(lambda s: [B.uint_dequant(up, uS, uZ, K, bits, G, B.UINT_NAIVE, out=out, stream=s) for _ in range(reps)])
-                tp, tf, tn = [min(time_graph(g, 5, 3) for _ in range(3)) / reps for g in (gp, gf, gn)]
                 nb = N * K * bits // 8 + N * (K // G) * 2 + N * K * 2
-                rows.append({"N": N, "K": K, "bits": bits, "G": G, "pot_us": tp * 1e3, "pot_Gweights_s": N * K / tp / 1e6,
-                             "pot_GBps": nb / tp / 1e6, "pot_frac_hbm": nb / tp / 1e6 / hbm, "uint_fast_us": tf * 1e3,
-                             "uint_naive_us": tn * 1e3, "pot_speedup_vs_best_uint": min(tf, tn) / tp})
-                del gp, gf, gn
-        del W, out
+                R = max(2, int(4 * L2_BYTES / nb) + 1)
+                outs = [torch.empty((N, K), dtype=torch.float16, device=dev) for _ in range(R)]
+                pk = [packed] + [packed.clone() for _ in range(R - 1)]
+                uk = [up] + [up.clone() for _ in range(R - 1)]
+                run_p = lambda i, s: B.pot_dequant(pk[i], S, K, bits, G, B.F16, out=outs[i], stream=s)
+                run_f = lambda i, s: B.uint_dequant(uk[i], uS, uZ, K, bits, G, B.UINT_FAST, out=outs[i], stream=s)
+                run_n = lambda i, s: B.uint_dequant(uk[i], uS, uZ, K, bits, G, B.UINT_NAIVE, out=outs[i], stream=s)
+                tp, tf, rf = ab_ratio(run_p, run_f, R, reps=5)
+                gn = capture(lambda s: [run_n(i, s) for i in range(R)])
+                tn = min(time_graph(gn, 3, 1) for _ in range(2)) / R
+                gw = capture(lambda s: [run_p(0, s) for _ in range(R)])
+                tw = min(time_graph(gw, 3, 1) for _ in range(2)) / R
+                rows.append({"N": N, "K": K, "bits": bits, "G": G, "rotating_pairs": R, "pot_us": tp * 1e3, "pot_Gweights_s": N * K / tp / 1e6,
+                             "pot_GBps": nb / tp / 1e6, "pot_frac_hbm": nb / tp / 1e6 / hbm, "pot_frac_8TBs_nominal": nb / tp / 1e6 / 8000.0,
+                             "uint_fast_us": tf * 1e3, "uint_naive_us": tn * 1e3, "uint_fast_over_pot_time": rf,
+                             "pot_us_l2_warm_same_buffers": tw * 1e3})
+                del outs, pk, uk, gn, gw
+                torch.cuda.empty_cache()
+        del W
         torch.cuda.empty_cache()
     ex["dequant_sweep"] = rows
+
+    # Algorithm 1 on the GPU (scale search, 200 candidates per group), set-up code: time per matrix
+    W = f16(synth.weights(synth.rng_for(1, 4096 % 97), 4096, 4096, "normal"))
+    with torch.cuda.stream(stream):
+        B.pot_quantize_ref(W, 3, GROUP, B.SCALE_SEARCH, stream=stream)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(3):
+            B.pot_quantize_ref(W, 3, GROUP, B.SCALE_SEARCH, stream=stream)
+        e1.record(stream)
+        stream.synchronize()
+    ta1 = e0.elapsed_time(e1) / 3
+    ex["algorithm1_scale_search_4096x4096_3bit"] = {"ms": ta1, "Mgroups_s": 4096 * 32 / ta1 / 1e3,
+                                                    "G_candidate_weight_evaluations_s": 4096 * 4096 * 200 / ta1 / 1e6}
+    del W
+    torch.cuda.empty_cache()
 
     # small-batch GEMM (config 4), HBM-cold
     rows = []
