@@ -227,9 +227,9 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
 /*
  * pot_gemm -- the matrix product that the dequantized weights feed (Sec. 4.2, last paragraph; reconstruction by
  * Eq. 1, decode by the integer add of Sec. 4.2): Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
- * accumulation, FP16 output.  M <= 6 (decode batches; also M = 7, 8 on shapes whose 128-row
- * tiles would fill the SMs badly) runs a tensor-core kernel that decodes weights straight into
- * MMA fragments; larger M runs the tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
+ * accumulation, FP16 output.  M <= 8 (decode batches) runs the streaming tensor-core kernel of
+ * pot_gemv with one token per MMA column, the weights decoded straight into MMA fragments;
+ * larger M runs the tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
  * accumulators in tensor memory (two issuing threads with an accumulator each, added in a fixed
  * order: the result does not depend on timing); the tiles of a last, at most half-filled wave
  * of CTAs -- or all tiles when they cover at most half of the SMs -- are split along K (FP32

@@ -1,7 +1,6 @@
 // pot_gemm: Y[M,N] = X[M,K] W~^T with the dequantization fused in.
 //
-//  * M <= 6 (and 7, 8 where the tcgen05 kernel's tiles would fill the SMs badly), tiled layout: tensor-core kernel on
-//    the shared-memory ring (ring.cuh).  The weights are the MMA's
+//  * M <= 8, tiled layout: the streaming tensor-core kernel of stream.cuh.  The weights are the MMA's
 //    M-side operand (16 rows per warp-step), the tokens its 8-wide N side, so no padding of M
 //    to 16 is needed and a warp decodes each record exactly once, straight into the A
 //    fragment registers -- the FP16 weights never exist in shared or global memory.
@@ -113,21 +112,18 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s);
 size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int bits, int group);
 bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group);
-double gemm_prefill_wave_fill(int64_t M, int64_t N, int64_t K);
 
 }  // namespace pot
 
 using namespace pot;
 
-// The streaming kernel (weights decoded straight into MMA fragments) serves up to 8 tokens and its time grows with
-// the batch; the tcgen05 kernel's time is flat in the batch but has a higher floor and works in 128-feature tiles.
-// Measured cross-over: up to 6 tokens the streaming kernel wins everywhere; at 7 and 8 tokens the tcgen05 kernel wins
-// (by 15 - 25 %) unless its tiles fill the SMs badly (e.g. 86 or 96 tiles on 148 SMs: 10 % slower).
-constexpr int64_t kSmallBatchMax = 8, kSmallBatchAlways = 6;
-constexpr double kMinWaveFill = 0.70;
+// The streaming kernel (weights decoded straight into MMA fragments, one token per MMA column) serves up to 8 tokens;
+// the tcgen05 kernel's time is flat in the batch but its floor is higher.  Measured on the 13B shapes: 13 - 23 us for
+// 1 - 8 tokens on the streaming kernel, 25 - 26 us for 8 - 32 tokens on the tcgen05 kernel.
+constexpr int64_t kSmallBatchMax = 8;
 static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout) {
-    if (layout != POT_LAYOUT_TILED || M > kSmallBatchMax || N % 16 != 0) return false;
-    return M <= kSmallBatchAlways || gemm_prefill_wave_fill(M, N, K) < kMinWaveFill;
+    (void)K;
+    return layout == POT_LAYOUT_TILED && M <= kSmallBatchMax && N % 16 == 0;
 }
 
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {

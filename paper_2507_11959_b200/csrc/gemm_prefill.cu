@@ -487,13 +487,6 @@ static PrefillPlan prefill_plan(int64_t M, int64_t N, int64_t K) {
     p.ws_bytes = tail ? p.counter_bytes + (size_t)tail * (size_t)s * (size_t)p.rows_alloc * PF_BN * 4 : 0;
     return p;
 }
-// share of the CTA slots that the kernel's work items fill, counted over whole waves (1.0 = every wave is full)
-double gemm_prefill_wave_fill(int64_t M, int64_t N, int64_t K) {
-    const PrefillPlan p = prefill_plan(M, N, K);
-    const int items = p.n_full + p.n_tail * p.splits;
-    const int waves = (items + kSmCount - 1) / kSmCount;
-    return waves > 0 ? (double)items / ((double)waves * kSmCount) : 0.0;
-}
 // arrival counters (must start at zero; the kernel leaves them at zero) + FP32 partial sums of the split tiles
 size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) { return prefill_plan(M, N, K).ws_bytes; }
 

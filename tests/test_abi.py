@@ -47,9 +47,9 @@ def test_size_helpers(L):
     assert ws >= 1024 + 256 * 2 * 16 * 4 and ws % 16 == 0
     wg = L.pot_gemm_workspace_bytes(6, 4096, 11008, 3, 128)   # small batch: eight token columns per slot
     assert wg >= 1024 + 256 * 2 * 16 * 8 * 4 and wg % 16 == 0
-    # 7 and 8 tokens: the streaming kernel only where the tcgen05 kernel's tiles would fill the SMs badly (96 tiles on 148)
+    # up to 8 tokens run the streaming kernel: one workspace size for all of them
     assert L.pot_gemm_workspace_bytes(8, 12288, 4096, 3, 128) == L.pot_gemm_workspace_bytes(6, 12288, 4096, 3, 128)
-    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 256 + 32 * 4 * 8 * 128 * 4
+    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == wg
     # Larger M runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
     # cover at most half of the SMs (32 tiles -> 4 splits of 32 token rows x 128 features), or those of a last
     # wave that fills at most half of the 148 CTA slots (640 tiles -> 48 tail tiles x 3 splits x 256 rows).
