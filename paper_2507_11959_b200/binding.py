@@ -11,8 +11,11 @@ from pathlib import Path
 
 import torch
 
+import os
+
 _HERE = Path(__file__).resolve().parent
-LIB_PATH = _HERE / "libpot_b200.so"
+# POT_B200_LIB selects another build of the same library (e.g. libpot_b200_checked.so, the -DPOT_CHECKED build)
+LIB_PATH = Path(os.environ["POT_B200_LIB"]) if os.environ.get("POT_B200_LIB") else _HERE / "libpot_b200.so"
 
 POT_OK = 0
 F16, BF16 = 0, 1

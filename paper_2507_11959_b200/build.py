@@ -13,6 +13,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libpot_b200.so"
+LIB_CHECKED = HERE / "libpot_b200_checked.so"   # the same sources with -DPOT_CHECKED (device-side index checks)
 OBJ_DIR = HERE / "build"
 SOURCES = ["api.cu", "quantize.cu", "dequant.cu", "gemv.cu", "gemm.cu", "gemm_prefill.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -31,13 +32,17 @@ def _deps_mtime() -> float:
     return max(f.stat().st_mtime for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> Path:
+    """Build the library; checked=True builds the variant whose kernels verify their indices before every store,
+    atomic and streamed shared-memory read and report a violation through the error words instead of accessing."""
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
+    OBJ_DIR = HERE / ("build_checked" if checked else "build")
     sources = [s for s in SOURCES if (CSRC / s).exists()]
     if not force and LIB.exists() and LIB.stat().st_mtime >= _deps_mtime():
         return LIB
     OBJ_DIR.mkdir(exist_ok=True)
     nvcc = _nvcc()
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"] + (["-DPOT_CHECKED"] if checked else [])
     flags += os.environ.get("POT_NVCC_FLAGS", "").split()  # extra compiler flags (experiments)
     if verbose:
         flags += ["-Xptxas", "-v"]
@@ -65,4 +70,4 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checked="--checked" in sys.argv))

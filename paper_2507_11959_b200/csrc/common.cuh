@@ -93,6 +93,18 @@ __device__ __forceinline__ uint32_t signed_exponent(uint32_t c, int ebit) {
     return e | s;
 }
 
+// Checked build (-DPOT_CHECKED): device-side index checks in front of stores, atomics and the streaming kernels'
+// shared-memory reads.  A failed check records `code` in the kernel family's error word (first failure wins) and the
+// access is skipped; nothing traps.  In the normal build the checks compile to nothing.
+#ifdef POT_CHECKED
+__device__ __forceinline__ bool in_range(bool ok, int* err, int code) {
+    if (!ok && err) atomicCAS(err, 0, code);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool in_range(bool, int*, int) { return true; }
+#endif
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif

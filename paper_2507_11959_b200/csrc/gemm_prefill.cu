@@ -367,7 +367,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             } else {
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             }
-            if (feat < N) {
+            if (feat < N && in_range(m0 + col < M && m0 >= 0 && feat >= 0 && (splits == 1 || (tail_index >= 0 && zsplit >= 0 && zsplit < splits)), err, 0x60)) {
                 if (splits == 1) {  // a warp stores 32 consecutive features (64 bytes) of one token at a time
                     __half* dst = Y + (m0 + col) * N + feat;
 #pragma unroll
@@ -381,7 +381,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 }
             }
         }
-        if (splits > 1) {
+        if (splits > 1 && in_range(tail_index >= 0 && partial != nullptr && counters != nullptr, err, 0x61)) {
             // The CTA that delivers the last split of a tile (an arrival counter tells it) adds the splits in
             // ascending order -- the result does not depend on timing -- and writes Y.
             __shared__ unsigned s_prev;

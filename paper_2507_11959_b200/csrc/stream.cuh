@@ -209,6 +209,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         const uint32_t left_j = n - j * SK_Q;
         const uint32_t cnt = left_j < (uint32_t)SK_Q ? left_j : (uint32_t)SK_Q;
         const uint32_t bar = bars + s * 8u, dst = ring + s * slot_bytes;
+        if (!in_range(s < (uint32_t)S && a + j * SK_Q + cnt <= sa.units && cnt >= 1, err, 0x110)) return;
         mbar_expect_tx(bar, cnt * (UB + NPARAM * PB));
         bulk_g2s(dst, pk + (size_t)j * (SK_Q * UB), cnt * UB, bar);
         bulk_g2s(dst + SK_Q * UB, ps + (size_t)j * SK_Q * PB, cnt * PB, bar);
@@ -287,7 +288,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         const int64_t row0 = (int64_t)rbd * 16;
         if (expect == 0) {
             if constexpr (TOK == 1) {
-                if (tig == 0) {
+                if (tig == 0 && in_range(row0 + gid + 8 < sa.N, err, 0x120)) {
                     sa.Y[row0 + gid] = __float2half_rn(v[0]);
                     sa.Y[row0 + gid + 8] = __float2half_rn(v[2]);
                 }
@@ -295,7 +296,8 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int token = 2 * tig + (e & 1);
-                    if (token < sa.M) sa.Y[(int64_t)token * sa.N + row0 + gid + 8 * (e >> 1)] = __float2half_rn(v[e]);
+                    if (token < sa.M && in_range(row0 + gid + 8 * (e >> 1) < sa.N, err, 0x121))
+                        sa.Y[(int64_t)token * sa.N + row0 + gid + 8 * (e >> 1)] = __float2half_rn(v[e]);
                 }
             }
             return;
@@ -303,6 +305,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         if (rbd == rb0 ? loc0 : locL) {
             // slot of warp w: [w][1] if w is the row block's first contributor, else [w][0]
             const uint32_t wl = (uint32_t)warp - slot;  // first contributor (local warp index)
+            if (!in_range(slot <= (uint32_t)warp && wl + expect <= (uint32_t)W && row0 + 16 <= sa.N, err, 0x130)) return;
             float* mine = lslots + ((size_t)warp * 2 + (slot == 0 ? 1 : 0)) * (16 * TOK);
             if constexpr (TOK == 1) {
                 if (tig == 0) {
@@ -328,6 +331,9 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             }
             return;
         }
+        if (!in_range(rbd < (uint32_t)sa.nrb && slot < (uint32_t)sa.max_slots && expect <= (uint32_t)sa.max_slots && sa.partial != nullptr,
+                      err, 0x140))
+            return;
         float* base = sa.partial + ((size_t)rbd * (size_t)sa.max_slots) * (16 * TOK);
         float* mine = base + (size_t)slot * (16 * TOK);
         if constexpr (TOK == 1) {
@@ -360,6 +366,10 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
 
     // ---- one unit: 2 x 32 codes of this lane -> 32 half2 -> eight MMAs ----------------------------------------
     auto unit = [&](const unsigned char* code, const unsigned char* param, uint32_t cbu) {
+        if (!in_range(code >= ringp && code + UB <= ringp + (size_t)S * slot_bytes && param + NPARAM * PB <= ringp + (size_t)S * slot_bytes &&
+                          cbu < ncb && (!XSMEM || (size_t)(cbu + 1) * 256u * (TOK == 1 ? 1 : 8) <= (size_t)sa.x_bytes),
+                      err, 0x150))
+            return;
         // activations of quarter tig (of token gid): the B fragments of the eight MMAs
         uint32_t xq[16];
         if constexpr (XSMEM) {

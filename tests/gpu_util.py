@@ -131,6 +131,8 @@ class GuardedBinding:
         torch.cuda.synchronize()
         for g in guards:
             assert g is None or g.intact(), f"{what}: a write landed outside its buffer"
+        # bounded waits that gave up, or (checked build) an index check that failed, leave a code in these words
+        assert self._b.pot_debug_errors() == (0, 0, 0), what
 
     def _ws(self, nbytes):
         return Guarded((nbytes,), torch.uint8, zero=True) if nbytes else None
