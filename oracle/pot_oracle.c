@@ -24,6 +24,8 @@
  * arithmetic, numpy's independent half conversion, numpy matmul, hand-derived fixtures,
  * invariants, and the integer-add formulation of Sec. 4.2 as an independent route).
  * po_scale_search (Algorithm 1) is pinned by brute force and by its optimality invariant.
+ * po_matmul_bf16 (the contraction on the BF16 reconstruction, BF16 activations) is pinned by numpy
+ * on float32-view conversions and a closed form.
  */
 #include <math.h>
 #include <stdint.h>
@@ -313,6 +315,50 @@ int po_matmul(const uint8_t* packed, const uint16_t* S, int64_t N, int64_t K, in
                 double y = 0.0, a = 0.0;
                 for (int64_t k = 0; k < K; ++k) {
                     double p = wrow[k] * po_f16_to_f64(X[m * K + k]);
+                    y += p;
+                    a += fabs(p);
+                }
+                Y[m * n_rows + r] = y;
+                A[m * n_rows + r] = a;
+            }
+        }
+        free(wrow);
+    }
+    return status;
+}
+
+/*
+ * The same contraction on the BF16 reconstruction with BF16 activations: w~ = (-1)^sign 2^E bf16_rne(S) (the paper's
+ * Sec. 4.2 is FP16-only; BF16 is this build's extension of the same integer add at exponent bit 7, with the scale
+ * rounded once to BF16), x[m,k] BF16 bit patterns, FP64 sums in the order k ascending.
+ */
+int po_matmul_bf16(const uint8_t* packed, const uint16_t* S, int64_t N, int64_t K, int bits, int G,
+                   const uint16_t* X, int64_t M, const int64_t* rows, int64_t n_rows,
+                   double* Y, double* A) {
+    if (!po_args_ok(N, K, bits, G) || M < 0 || n_rows < 0) return -1;
+    if (!rows && n_rows != N) return -1;
+    const int64_t row_bytes = K * bits / 8, ng = K / G;
+    int status = 0;
+#pragma omp parallel
+    {
+        double* wrow = (double*)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1));
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            int64_t i = rows ? rows[r] : r;
+            if (i < 0 || i >= N || !wrow) {
+#pragma omp atomic write
+                status = -1;
+                continue;
+            }
+            const uint8_t* row = packed + i * row_bytes;
+            for (int64_t k = 0; k < K; ++k) {
+                double v = po_value(po_code_at(row, k, bits), S[i * ng + k / G], bits, PO_BF16);
+                wrow[k] = po_bf16_to_f64(po_f64_to_bf16(v, NULL));
+            }
+            for (int64_t m = 0; m < M; ++m) {
+                double y = 0.0, a = 0.0;
+                for (int64_t k = 0; k < K; ++k) {
+                    double p = wrow[k] * po_bf16_to_f64(X[m * K + k]);
                     y += p;
                     a += fabs(p);
                 }

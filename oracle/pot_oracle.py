@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.po_dequant.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp]
         L.po_matmul.restype = i32
         L.po_matmul.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp, i64, vp, vp]
+        L.po_matmul_bf16.restype = i32
+        L.po_matmul_bf16.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp, i64, vp, vp]
         L.po_scale_search.restype = i32
         L.po_scale_search.argtypes = [vp, i64, i64, i32, i32, vp, vp]
         L.pu_quantize.restype = i32
@@ -164,8 +166,9 @@ def dequant(packed: np.ndarray, scales: np.ndarray, K: int, bits: int, G: int,
 
 
 def matmul(packed: np.ndarray, scales: np.ndarray, K: int, bits: int, G: int, X_bits: np.ndarray,
-           rows: np.ndarray | None = None) -> tuple[np.ndarray, np.ndarray]:
-    """FP64 Y [M, n_rows] and A = sum|w*x| [M, n_rows] on the FP16 reconstruction."""
+           rows: np.ndarray | None = None, dtype: int = F16) -> tuple[np.ndarray, np.ndarray]:
+    """FP64 Y [M, n_rows] and A = sum|w*x| [M, n_rows] on the FP16 reconstruction with FP16 activations (dtype F16) or
+    on the BF16 reconstruction with BF16 activations (dtype BF16; X_bits are then BF16 bit patterns)."""
     packed = _c(packed, np.uint8)
     scales = _c(scales, np.uint16)
     X_bits = _c(X_bits, np.uint16).reshape(-1, K)
@@ -175,7 +178,8 @@ def matmul(packed: np.ndarray, scales: np.ndarray, K: int, bits: int, G: int, X_
     n_rows = N if rows is None else rows.shape[0]
     Y = np.zeros((M, n_rows), dtype=np.float64)
     A = np.zeros((M, n_rows), dtype=np.float64)
-    rc = lib().po_matmul(_p(packed), _p(scales), N, K, bits, G, _p(X_bits), M, _p(rows), n_rows, _p(Y), _p(A))
+    fn = lib().po_matmul if dtype == F16 else lib().po_matmul_bf16
+    rc = fn(_p(packed), _p(scales), N, K, bits, G, _p(X_bits), M, _p(rows), n_rows, _p(Y), _p(A))
     if rc != 0:
         raise ValueError(f"po_matmul failed with {rc}")
     return Y, A

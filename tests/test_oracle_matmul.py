@@ -67,3 +67,39 @@ def test_matmul_rows_equal_separate_gemvs(oracle):
     for m in range(M):
         y1, a1 = oracle.matmul(packed, S, K, bits, G, X[m:m + 1])
         assert np.array_equal(y1[0], Y[m]) and np.array_equal(a1[0], A[m])
+
+
+def _bf16_bits_to_f64(bits):
+    """BF16 bit patterns -> FP64 through numpy's float32 view (independent of the oracle's own conversion)"""
+    return (np.ascontiguousarray(bits).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _f16_bits_to_bf16_bits(bits):
+    """round-to-nearest-even FP16 -> BF16 by integer arithmetic on the float32 pattern"""
+    u = np.ascontiguousarray(bits).view(np.float16).astype(np.float32).view(np.uint32)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("bits,G", [(2, 128), (3, 128), (4, 64), (3, 64)])
+def test_bf16_matmul_matches_numpy(oracle, bits, G):
+    """The BF16 contraction against numpy on the oracle's BF16 dequantization (itself pinned in test_oracle_formats),
+    with activations rounded to BF16 by independent integer arithmetic; and a closed form: codes 0, x = 1."""
+    N, K, M = 64, 768, 3
+    packed, S, X16 = _case(oracle, bits, G, N, K, M, seed=10 + bits)
+    Xb = _f16_bits_to_bf16_bits(X16)
+    deq, rounded = oracle.dequant(packed, S, K, bits, G, oracle.BF16)
+    assert rounded == 0
+    w, x = _bf16_bits_to_f64(deq), _bf16_bits_to_f64(Xb)
+    Y, A = oracle.matmul(packed, S, K, bits, G, Xb, dtype=oracle.BF16)
+    ref, refA = x @ w.T, np.abs(x) @ np.abs(w).T
+    assert np.allclose(Y, ref, rtol=0, atol=1e-12 * refA.max()) and np.allclose(A, refA, rtol=1e-13, atol=0)
+    # it is not the FP16 contraction: the scale is rounded to 8 significant bits first
+    Y16, _ = oracle.matmul(packed, S, K, bits, G, X16)
+    assert not np.allclose(Y, Y16, rtol=1e-6, atol=0)
+    # all codes 0 (sign +, E = 0), x = 1: y_i = G * sum_g bf16(S_ig), exactly
+    z = np.zeros((4, 256 * bits // 8), dtype=np.uint8)
+    S2 = np.array([[0x2E66, 0x3555]] * 4, dtype=np.uint16)       # bf16: 0x3DCD, 0x3EAB
+    ones = np.full((1, 256), 0x3F80, dtype=np.uint16)
+    Y1, _ = oracle.matmul(z, S2, 256, bits, 128, ones, dtype=oracle.BF16)
+    expect = 128 * (_bf16_bits_to_f64(np.array([0x3DCD], dtype=np.uint16))[0] + _bf16_bits_to_f64(np.array([0x3EAB], dtype=np.uint16))[0])
+    assert np.all(Y1 == expect)
