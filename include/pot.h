@@ -191,6 +191,18 @@ pot_status_t pot_gemv(const void* packed, const void* scales_f16, int64_t N, int
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * pot_gemv_bf16 -- pot_gemv with BF16 activations, BF16 reconstruction and BF16 output.  The paper's kernel (Sec. 4.2)
+ * is written for FP16; the same integer add applies to BF16 with the exponent at bit 7: the group's FP16 scale is
+ * rounded once to BF16 (round to nearest even) and E is added to that pattern, w~ = +-2^E * bf16(S) exactly, as in
+ * pot_dequant with POT_BF16.  x_bf16 [K], y_bf16 [N]; everything else as pot_gemv (same layouts, same workspace).
+ * In the tiled layout the codes keep their FP16-shaped bit map, so the BF16 decode needs two mask / multiply-add
+ * pairs per register where FP16 needs one: expect a slower kernel at equal bytes.
+ */
+pot_status_t pot_gemv_bf16(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                           int group, pot_layout_t layout, const void* x_bf16, void* y_bf16,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * pot_gemv_host -- pot_gemv for a caller whose activations and results live in HOST memory
  * (ideally pinned): copies x_host [K] to d_x, runs pot_gemv, copies the result to y_host [N],
  * all asynchronously on `stream`.  The weights stay resident on the device.
@@ -241,6 +253,13 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
 pot_status_t pot_gemm(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
                       int group, pot_layout_t layout, const void* X_f16, int64_t M, void* Y_f16,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* pot_gemm_bf16 -- pot_gemm with BF16 activations X_bf16 [M,K], BF16 reconstruction (see pot_gemv_bf16) and BF16
+ * output Y_bf16 [M,N]; same routes (streaming kernel, tcgen05 kernel with the BF16 instruction kind, canonical
+ * fallback), same workspace sizes.                                                                              */
+pot_status_t pot_gemm_bf16(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
+                           int group, pot_layout_t layout, const void* X_bf16, int64_t M, void* Y_bf16,
+                           void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---- uniform-INT (zero-point) twin at the same bits and group size ------------------------
  * The baseline the paper compares against (first equation of Sec. 4.1): w~ = (W_Q + Z) o S.

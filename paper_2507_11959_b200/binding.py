@@ -26,7 +26,7 @@ UINT_FAST, UINT_NAIVE = 0, 1
 EXPORTS = [
     "pot_status_string", "pot_packed_bytes", "pot_scales_bytes", "pot_gemv_workspace_bytes",
     "pot_gemm_workspace_bytes", "pot_launch_count", "pot_quantize_ref", "pot_validate_scales", "pot_repack", "pot_repack_scales", "pot_layout_scale_index",
-    "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_host", "pot_gemm", "uint_quantize_ref", "uint_dequant",
+    "uint_repack", "pot_dequant", "pot_gemv", "pot_gemv_bf16", "pot_gemv_host", "pot_gemm", "pot_gemm_bf16", "uint_quantize_ref", "uint_dequant",
     "uint_gemv", "pot_layout_bit", "pot_gemv_noalloc", "pot_gemv_noalloc_max_scratch_bytes", "pot_debug_gemv_error", "pot_debug_gemv_plan", "pot_debug_gemm_error", "pot_debug_prefill_error",
 ]
 
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.pot_layout_scale_index.argtypes = [i64, i64, i32, i64, i64, vp]
         L.pot_dequant.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.pot_gemv.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.pot_gemv_bf16.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.pot_gemm_bf16.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, i64, vp, vp, sz, vp]
         L.pot_gemv_host.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.pot_gemm.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, i64, vp, vp, sz, vp]
         L.uint_quantize_ref.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp]
@@ -194,14 +196,18 @@ def pot_dequant(packed: torch.Tensor, scales: torch.Tensor, K: int, bits: int, g
 
 def pot_gemv(packed, scales, K: int, bits: int, group: int, x: torch.Tensor, layout: int = CANONICAL,
              y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """x float16 -> pot_gemv, x bfloat16 -> pot_gemv_bf16 (the output has the activations' dtype)."""
     N = packed.shape[0]
+    assert x.dtype in (torch.float16, torch.bfloat16)
     if y is None:
-        y = torch.empty(N, dtype=torch.float16, device=x.device)
+        y = torch.empty(N, dtype=x.dtype, device=x.device)
+    assert y.dtype == x.dtype
     need = pot_gemv_workspace_bytes(N, K, bits, group) if layout == TILED else 0
     if need and workspace is None:
         workspace = new_workspace(need, x.device)
-    _check(lib().pot_gemv(_ptr(packed), _ptr(scales), N, K, bits, group, layout, _ptr(x), _ptr(y), _ptr(workspace),
-                          0 if workspace is None else workspace.numel(), _stream(stream)), "pot_gemv")
+    fn = lib().pot_gemv if x.dtype == torch.float16 else lib().pot_gemv_bf16
+    _check(fn(_ptr(packed), _ptr(scales), N, K, bits, group, layout, _ptr(x), _ptr(y), _ptr(workspace),
+              0 if workspace is None else workspace.numel(), _stream(stream)), "pot_gemv")
     return y
 
 
@@ -218,13 +224,16 @@ def pot_gemv_host(packed, scales, K: int, bits: int, group: int, x_host: torch.T
 def pot_gemm(packed, scales, K: int, bits: int, group: int, X: torch.Tensor, layout: int = CANONICAL,
              Y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
     N, M = packed.shape[0], X.shape[0]
+    assert X.dtype in (torch.float16, torch.bfloat16)
     if Y is None:
-        Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+        Y = torch.empty((M, N), dtype=X.dtype, device=X.device)
+    assert Y.dtype == X.dtype
     need = pot_gemm_workspace_bytes(M, N, K, bits, group) if layout == TILED else 0
     if need and workspace is None:
         workspace = new_workspace(need, X.device)
-    _check(lib().pot_gemm(_ptr(packed), _ptr(scales), N, K, bits, group, layout, _ptr(X), M, _ptr(Y), _ptr(workspace),
-                          0 if workspace is None else workspace.numel(), _stream(stream)), "pot_gemm")
+    fn = lib().pot_gemm if X.dtype == torch.float16 else lib().pot_gemm_bf16
+    _check(fn(_ptr(packed), _ptr(scales), N, K, bits, group, layout, _ptr(X), M, _ptr(Y), _ptr(workspace),
+              0 if workspace is None else workspace.numel(), _stream(stream)), "pot_gemm")
     return Y
 
 

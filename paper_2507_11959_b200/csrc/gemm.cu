@@ -21,11 +21,12 @@ namespace pot {
 // ------------------------------------------------------------------------------------------
 constexpr int FB_LD = 136;  // padded leading dimension (halves) -> conflict-free fragment loads
 
-template <int BITS>
+template <int BITS, int DT = 0>  // DT = 1: BF16 activations, weights (scale rounded once to BF16) and output
 __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* __restrict__ packed,
                                                                 const uint16_t* __restrict__ scales, int64_t N, int64_t K,
                                                                 int G, const __half* __restrict__ X, int64_t M,
-                                                                __half* __restrict__ Y) {
+                                                                uint16_t* __restrict__ Y) {
+    constexpr int EBIT = DT == 0 ? 10 : 7;
     constexpr uint32_t CM = (1u << BITS) - 1u;
     constexpr uint32_t QM2 = (uint32_t)qmax_of(BITS) * 0x10001u;
     constexpr uint32_t SM2 = (1u << (BITS - 1)) * 0x10001u;
@@ -56,13 +57,15 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
             if (row < N) {
                 const int64_t k = kb * 128 + pc * 8;
                 const uint32_t v = read_bits(packed + row * (K * BITS / 32), k * BITS, 8 * BITS);
-                const uint32_t sc2 = (uint32_t)__ldg(scales + row * (K / G) + k / G) * 0x10001u;
+                uint32_t s16 = __ldg(scales + row * (K / G) + k / G);
+                if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
+                const uint32_t sc2 = s16 * 0x10001u;
                 uint32_t o[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t t = v >> (2 * j * BITS);
                     const uint32_t pr = (t & CM) | ((t << (16 - BITS)) & (CM << 16));
-                    o[j] = sc2 + (((pr & QM2) << 10) | ((pr & SM2) << (16 - BITS)));
+                    o[j] = sc2 + (((pr & QM2) << EBIT) | ((pr & SM2) << (16 - BITS)));
                 }
                 wv = make_uint4(o[0], o[1], o[2], o[3]);
             }
@@ -90,7 +93,10 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
 #pragma unroll
             for (int i = 0; i < 2; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) sk_mma(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
+                for (int j = 0; j < 4; ++j) {
+                    if (DT == 0) sk_mma(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
+                    else sk_mma_bf16(acc[i][j], a[i][0], a[i][1], a[i][2], a[i][3], b[j][0], b[j][1]);
+                }
         }
     }
 #pragma unroll
@@ -102,14 +108,14 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
                 const int64_t token = m0 + wm + 16 * i + gid + 8 * hh;
                 const int64_t row = n0 + wn + 8 * j + 2 * tig;
                 if (token < M) {
-                    if (row < N) Y[token * N + row] = __float2half_rn(acc[i][j][2 * hh]);
-                    if (row + 1 < N) Y[token * N + row + 1] = __float2half_rn(acc[i][j][2 * hh + 1]);
+                    if (row < N) Y[token * N + row] = sk_out<DT>(acc[i][j][2 * hh]);
+                    if (row + 1 < N) Y[token * N + row + 1] = sk_out<DT>(acc[i][j][2 * hh + 1]);
                 }
             }
 }
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
-                                 const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s);
+                                 const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s, int dt);
 size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int bits, int group);
 bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group);
 
@@ -132,9 +138,10 @@ extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int 
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
-extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
-                                 pot_layout_t layout, const void* X, int64_t M, void* Y, void* workspace,
-                                 size_t ws_bytes, void* stream) {
+template <int DT>
+static pot_status_t gemm_impl(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                              pot_layout_t layout, const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes,
+                              void* stream) {
     if (!packed || !scales || !X || !Y) return POT_ERR_NULL;
     pot_status_t st = check_shape(N, K, bits, group);
     if (st != POT_OK) return st;
@@ -148,7 +155,7 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
         const size_t need = pot_gemm_workspace_bytes(M, N, K, bits, group);
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
         const int Mi = (int)M;
-#define POT_GS(B) return launch_stream<B, SK_POT, 8, 16>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, error_ptr(ERR_GEMM), s)
+#define POT_GS(B) return launch_stream<B, SK_POT, 8, 16, 1, DT>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, error_ptr(ERR_GEMM), s)
         if (bits == 2) POT_GS(2);
         if (bits == 3) POT_GS(3);
         POT_GS(4);
@@ -156,14 +163,27 @@ extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t
     }
     if (layout == POT_LAYOUT_TILED) {
         if (!gemm_prefill_supported(M, N, K, bits, group)) return POT_ERR_UNSUPPORTED;
-        return gemm_prefill_launch(packed, scales, N, K, bits, group, X, M, Y, workspace, ws_bytes, s);
+        return gemm_prefill_launch(packed, scales, N, K, bits, group, X, M, Y, workspace, ws_bytes, s, DT);
     }
+    if ((M + 63) / 64 > 65535) return POT_ERR_SHAPE;  // the fallback kernel's token tiles ride on gridDim.y
     const dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64)), block(128);
     auto* P = (const uint32_t*)packed;
     auto* S = (const uint16_t*)scales;
-    if (bits == 2) return launch_pdl(pot_gemm_fallback_kernel<2>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (__half*)Y);
-    if (bits == 3) return launch_pdl(pot_gemm_fallback_kernel<3>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (__half*)Y);
-    return launch_pdl(pot_gemm_fallback_kernel<4>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (__half*)Y);
+    if (bits == 2) return launch_pdl(pot_gemm_fallback_kernel<2, DT>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (uint16_t*)Y);
+    if (bits == 3) return launch_pdl(pot_gemm_fallback_kernel<3, DT>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (uint16_t*)Y);
+    return launch_pdl(pot_gemm_fallback_kernel<4, DT>, grid, block, 0, s, P, S, N, K, group, (const __half*)X, M, (uint16_t*)Y);
+}
+
+extern "C" pot_status_t pot_gemm(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                 pot_layout_t layout, const void* X, int64_t M, void* Y, void* workspace,
+                                 size_t ws_bytes, void* stream) {
+    return gemm_impl<0>(packed, scales, N, K, bits, group, layout, X, M, Y, workspace, ws_bytes, stream);
+}
+
+extern "C" pot_status_t pot_gemm_bf16(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                      pot_layout_t layout, const void* X, int64_t M, void* Y, void* workspace,
+                                      size_t ws_bytes, void* stream) {
+    return gemm_impl<1>(packed, scales, N, K, bits, group, layout, X, M, Y, workspace, ws_bytes, stream);
 }
 
 // Diagnostic: reads and clears the device error word of the gemm kernels in this library (0 = every bounded

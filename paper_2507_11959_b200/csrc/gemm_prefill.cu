@@ -53,8 +53,17 @@ constexpr size_t pf_smem_bytes(int stages, int mt) { return 1024 /*align slack*/
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128 (the weight rows of the tile are the
 // A operand), N = n token rows of the X tile (the B operand), 16 <= n <= 256, n % 16 == 0
-__host__ __device__ constexpr uint32_t pf_idesc(uint32_t n) {
-    return (1u << 4) /*D = F32*/ | (0u << 7) /*A = F16*/ | (0u << 10) /*B = F16*/ | ((n >> 3) << 17) | ((uint32_t)(PF_BN >> 4) << 24);
+// (dt = 1: BF16 x BF16 -> FP32)
+__host__ __device__ constexpr uint32_t pf_idesc(uint32_t n, uint32_t dt = 0) {
+    return (1u << 4) /*D = F32*/ | (dt << 7) /*A = F16 / BF16*/ | (dt << 10) /*B = F16 / BF16*/ | ((n >> 3) << 17) |
+           ((uint32_t)(PF_BN >> 4) << 24);
+}
+
+// FP32 sum -> FP16 (DT = 0) or BF16 (DT = 1) bit pattern, round to nearest even
+template <int DT>
+__device__ __forceinline__ uint16_t pf_out(float v) {
+    if (DT == 0) return __half_as_ushort(__float2half_rn(v));
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
 }
 
 // shared-memory matrix descriptor, K-major, 128-byte swizzle: start >> 4, LBO = 1 (unused), SBO = 1024 B
@@ -116,7 +125,7 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // high word is a constant); the loop is unrolled over the stages so that these stay in registers and a K step is one
 // add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the test for the issuer's
 // next stage is put in flight before the MMAs of this one are issued and examined afterwards.
-template <int J, int NI, int PF_STAGES, int MT>
+template <int J, int NI, int PF_STAGES, int MT, int DT = 0>
 __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, uint32_t n_tok, int* err) {
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
@@ -130,7 +139,7 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
     }
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
     const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BM * MT);   // this issuer's accumulator: 128 features x (128 MT) token columns
-    const uint32_t idesc = pf_idesc(n_tok);
+    const uint32_t idesc = pf_idesc(n_tok, DT);
     uint32_t ready = mbar_test(full(J), 0);
     uint32_t ph = 0;
     for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
@@ -161,11 +170,11 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
 // Instantiated as <bits, 4, 4, 2, 2> (M > 64: 256-token tiles, four 48 KB stages) and <bits, 8, 4, 2, 1> (M <= 64: one
 // tile of up to 64 tokens, eight 24 KB stages -- a stage buffer's round trip producer -> issuer -> tensor pipe ->
 // producer is ~2000 cycles whatever the tile holds, so more buffers = more stages per unit of time).
-template <int BITS, int PF_STAGES, int NG, int NI, int MT>
+template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0>  // DT = 1: BF16 activations, weights and output
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
-                        __half* __restrict__ Y, float* __restrict__ partial, unsigned* __restrict__ counters,
+                        uint16_t* __restrict__ Y, float* __restrict__ partial, unsigned* __restrict__ counters,
                         int tiles_m, int n_full, int tail_splits, int* __restrict__ err) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
@@ -260,8 +269,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
-            else pf_issue<NI - 1, NI, PF_STAGES, MT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
         }
     } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
@@ -316,12 +325,15 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     __syncwarp();
                 }
                 unsigned char* brow = smem + (size_t)s * STAGE_BYTES + pf_x_bytes(MT) + row * 128;
-                const uint32_t s2 = sc2[buf] * 0x10001u;  // scale pattern in both halves
+                uint32_t s16 = sc2[buf];
+                if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
+                const uint32_t s2 = s16 * 0x10001u;  // scale pattern in both halves
 #pragma unroll
                 for (int T2 = 0; T2 < 2; ++T2) {
                     uint32_t w2[16];
                     if (row_ok) {
-                        potl::pot_decode32<BITS, 2>(rec[buf], T2, s2, w2);
+                        if (DT == 0) potl::pot_decode32<BITS, 2>(rec[buf], T2, s2, w2);
+                        else potl::pot_decode32_bf16<BITS, 2>(rec[buf], T2, s2, w2);
                     } else {
 #pragma unroll
                         for (int q = 0; q < 16; ++q) w2[q] = 0u;
@@ -369,10 +381,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             }
             if (feat < N && in_range(m0 + col < M && m0 >= 0 && feat >= 0 && (splits == 1 || (tail_index >= 0 && zsplit >= 0 && zsplit < splits)), err, 0x60)) {
                 if (splits == 1) {  // a warp stores 32 consecutive features (64 bytes) of one token at a time
-                    __half* dst = Y + (m0 + col) * N + feat;
+                    uint16_t* dst = Y + (m0 + col) * N + feat;
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (m0 + col + i < M) dst[(int64_t)i * N] = __float2half_rn(__uint_as_float(v[i]));
+                        if (m0 + col + i < M) dst[(int64_t)i * N] = pf_out<DT>(__uint_as_float(v[i]));
                 } else {  // this split's partial sums: [tail tile][split][token of the tile][128 features] FP32
                     float* dst = partial + (((int64_t)tail_index * splits + zsplit) * rows_alloc + col) * PF_BN + (32 * q + lane);
 #pragma unroll
@@ -415,9 +427,9 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                         const int pc = p0 + u * NPT;
                         const int64_t row = m0 + pc / (PF_BN / 4), colx = n0 + 4 * (pc % (PF_BN / 4));
                         if (pc < npieces && row < M && colx < N) {  // N % 16 == 0: a piece is inside or outside as a whole
-                            const __half2 h0 = __floats2half2_rn(acc4[u].x, acc4[u].y), h1 = __floats2half2_rn(acc4[u].z, acc4[u].w);
-                            *reinterpret_cast<uint2*>(Y + row * N + colx) =
-                                make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                            const uint32_t h0 = (uint32_t)pf_out<DT>(acc4[u].x) | ((uint32_t)pf_out<DT>(acc4[u].y) << 16);
+                            const uint32_t h1 = (uint32_t)pf_out<DT>(acc4[u].z) | ((uint32_t)pf_out<DT>(acc4[u].w) << 16);
+                            *reinterpret_cast<uint2*>(Y + row * N + colx) = make_uint2(h0, h1);
                         }
                     }
                 }
@@ -493,7 +505,7 @@ size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) { retur
 static int* prefill_error_ptr();
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
-                                 const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s) {
+                                 const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s, int dt) {
     const PrefillPlan pl = prefill_plan(M, N, K);
     if (pl.ws_bytes > 0 && (!workspace || ws_bytes < pl.ws_bytes)) return POT_ERR_WORKSPACE;
     unsigned* counters = (unsigned*)workspace;
@@ -515,9 +527,19 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         const dim3 block((unsigned)pf_threads(4, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
-                          (__half*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
+                          (uint16_t*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
     // four producer groups, two issuers, one CTA per SM; one token tile and eight 24 KB stages for batches of up to 64 tokens
+    if (dt == 1) {
+        if (M <= PF_SMALL_TOKENS) {
+            if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1, 1>, 8, 1);
+            if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1, 1>, 8, 1);
+            return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1, 1>, 8, 1);
+        }
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2, 1>, 4, 2);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 1>, 4, 2);
+        return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 1>, 4, 2);
+    }
     if (M <= PF_SMALL_TOKENS) {
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1>, 8, 1);

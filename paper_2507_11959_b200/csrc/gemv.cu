@@ -33,11 +33,19 @@ __device__ __forceinline__ void rg_fma2(float& acc0, float& acc1, uint32_t w2, u
 // ------------------------------------------------------------------------------------------
 // canonical layout, one warp per row
 // ------------------------------------------------------------------------------------------
-template <int BITS, bool UNIFORM>
+// BF16 pairs: a BF16 number is the upper half of an FP32 pattern, so the conversions are a shift and a mask
+__device__ __forceinline__ void rg_fma2_bf16(float& acc0, float& acc1, uint32_t w2, uint32_t x2) {
+    acc0 = fmaf(__uint_as_float(w2 << 16), __uint_as_float(x2 << 16), acc0);
+    acc1 = fmaf(__uint_as_float(w2 & 0xFFFF0000u), __uint_as_float(x2 & 0xFFFF0000u), acc1);
+}
+
+// DT = 0: FP16 activations / weights / output; DT = 1: BF16 (PoT only: scale rounded once to BF16, E added at bit 7)
+template <int BITS, bool UNIFORM, int DT = 0>
 __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __restrict__ packed,
                                                              const uint16_t* __restrict__ scales,
                                                              const uint16_t* __restrict__ zeros, int64_t N, int64_t K,
-                                                             int G, const uint4* __restrict__ x, __half* __restrict__ y) {
+                                                             int G, const uint4* __restrict__ x, uint16_t* __restrict__ y) {
+    constexpr int EBIT = DT == 0 ? 10 : 7;
     constexpr uint32_t CM = (1u << BITS) - 1u;
     constexpr uint32_t QM2 = (uint32_t)qmax_of(BITS) * 0x10001u;
     constexpr uint32_t SM2 = (1u << (BITS - 1)) * 0x10001u;
@@ -52,7 +60,8 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
     pdl_wait();
     for (int64_t c = lane; c < pieces; c += 32) {
         const uint32_t v = read_bits(rowp, c * (8 * BITS), 8 * BITS);
-        const uint32_t s16 = __ldg(srow + (c * 8) / G);
+        uint32_t s16 = __ldg(srow + (c * 8) / G);
+        if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
         const uint4 xv = __ldg(x + c);
         const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
@@ -61,7 +70,7 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
             const uint32_t pr = (t & CM) | ((t << (16 - BITS)) & (CM << 16));
             uint32_t w2;
             if constexpr (!UNIFORM) {
-                w2 = s16 * 0x10001u + (((pr & QM2) << 10) | ((pr & SM2) << (16 - BITS)));
+                w2 = s16 * 0x10001u + (((pr & QM2) << EBIT) | ((pr & SM2) << (16 - BITS)));
             } else {
                 const __half2 zm2 = __hadd2(__half2half2(__ushort_as_half(__ldg(zrow + (c * 8) / G))), __float2half2_rn(1024.0f));
                 const uint32_t h = pr | 0x64006400u;
@@ -69,12 +78,13 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
                 const __half2 w = __hmul2(d, __half2half2(__ushort_as_half((uint16_t)s16)));
                 w2 = *reinterpret_cast<const uint32_t*>(&w);
             }
-            rg_fma2(acc0, acc1, w2, xs[j]);
+            if (DT == 0) rg_fma2(acc0, acc1, w2, xs[j]);
+            else rg_fma2_bf16(acc0, acc1, w2, xs[j]);
         }
     }
     float acc = acc0 + acc1;
     for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) y[row] = __float2half_rn(acc);
+    if (lane == 0) y[row] = sk_out<DT>(acc);
 }
 
 // CTAs per SM of the streaming GEMV (16 consumer warps each).  Two: the next launch in the stream becomes resident,
@@ -89,11 +99,11 @@ static int gemv_occupancy(int64_t N, int64_t K, int bits, int group, int kind) {
     return share <= kTwoCtaMaxShare ? 2 : 1;
 }
 
-template <int KIND>
+template <int KIND, int DT = 0>
 static pot_status_t launch_gemv_stream(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
                                        int bits, int group, const void* x, void* y, void* workspace, cudaStream_t s) {
     int* err = error_ptr(ERR_GEMV);
-#define POT_SG(B, O) return launch_stream<B, KIND, 1, 16, O>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s)
+#define POT_SG(B, O) return launch_stream<B, KIND, 1, 16, O, DT>(packed, scales, zeros, N, K, group, x, 1, y, workspace, err, s)
     if (gemv_occupancy(N, K, bits, group, KIND) == 2) {
         if (bits == 2) POT_SG(2, 2);
         if (bits == 3) POT_SG(3, 2);
@@ -160,9 +170,9 @@ static pot_status_t check_gemv_args(const void* packed, const void* scales, int6
     return POT_OK;
 }
 
-extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
-                                 pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes,
-                                 void* stream) {
+template <int DT>
+static pot_status_t gemv_impl(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                              pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes, void* stream) {
     const pot_status_t st = check_gemv_args(packed, scales, N, K, bits, group, layout, x, y, workspace, ws_bytes);
     if (st != POT_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
@@ -170,11 +180,24 @@ extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t
         const dim3 grid((unsigned)((N + 7) / 8)), block(256);
         auto* P = (const uint32_t*)packed;
         auto* S = (const uint16_t*)scales;
-        if (bits == 2) return launch_pdl(gemv_canonical_kernel<2, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
-        if (bits == 3) return launch_pdl(gemv_canonical_kernel<3, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
-        return launch_pdl(gemv_canonical_kernel<4, false>, grid, block, 0, s, P, S, (const uint16_t*)nullptr, N, K, group, (const uint4*)x, (__half*)y);
+        const uint16_t* Z = nullptr;
+        if (bits == 2) return launch_pdl(gemv_canonical_kernel<2, false, DT>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
+        if (bits == 3) return launch_pdl(gemv_canonical_kernel<3, false, DT>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
+        return launch_pdl(gemv_canonical_kernel<4, false, DT>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
     }
-    return launch_gemv_stream<SK_POT>(packed, scales, nullptr, N, K, bits, group, x, y, workspace, s);
+    return launch_gemv_stream<SK_POT, DT>(packed, scales, nullptr, N, K, bits, group, x, y, workspace, s);
+}
+
+extern "C" pot_status_t pot_gemv(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                 pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes,
+                                 void* stream) {
+    return gemv_impl<0>(packed, scales, N, K, bits, group, layout, x, y, workspace, ws_bytes, stream);
+}
+
+extern "C" pot_status_t pot_gemv_bf16(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
+                                      pot_layout_t layout, const void* x, void* y, void* workspace, size_t ws_bytes,
+                                      void* stream) {
+    return gemv_impl<1>(packed, scales, N, K, bits, group, layout, x, y, workspace, ws_bytes, stream);
 }
 
 extern "C" pot_status_t pot_gemv_host(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -207,9 +230,9 @@ extern "C" pot_status_t uint_gemv(const void* packed, const void* scales, const 
     if (layout == POT_LAYOUT_CANONICAL) {
         const dim3 grid((unsigned)((N + 7) / 8)), block(256);
         auto* P = (const uint32_t*)packed;
-        if (bits == 2) return launch_pdl(gemv_canonical_kernel<2, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (__half*)y);
-        if (bits == 3) return launch_pdl(gemv_canonical_kernel<3, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (__half*)y);
-        return launch_pdl(gemv_canonical_kernel<4, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (__half*)y);
+        if (bits == 2) return launch_pdl(gemv_canonical_kernel<2, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
+        if (bits == 3) return launch_pdl(gemv_canonical_kernel<3, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
+        return launch_pdl(gemv_canonical_kernel<4, true>, grid, block, 0, s, P, S, Z, N, K, group, (const uint4*)x, (uint16_t*)y);
     }
     if (N % 16 != 0) return POT_ERR_SHAPE;
     const size_t need = pot_gemv_workspace_bytes(N, K, bits, group);

@@ -190,6 +190,39 @@ __device__ __forceinline__ void pot_decode32(const uint32_t* rec, int T, uint32_
     }
 }
 
+// t * c (upper 32 bits of the product) + s as one instruction: a right shift by 32 - log2(c) fused with the add
+__device__ __forceinline__ uint32_t madhi(uint32_t t, uint32_t c, uint32_t s) {
+    uint32_t d;
+    asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(t), "r"(c), "r"(s));
+    return d;
+}
+
+// The same decode for BF16 (1 sign, 8 exponent, 7 mantissa bits): out[p] = bit pattern of bfloat162{ w~[2p], w~[2p+1] }
+// with w~ = +-2^E * bf16(S); sc2 holds the BF16-rounded scale in both halves.  The byte lanes were shaped for FP16 (sign
+// five positions above the exponent's low bit); in BF16 the exponent's low bit is bit 7 and the sign eight positions
+// above it, so exponent and sign are masked and aligned separately: two mask / multiply-add pairs per register instead
+// of one (for the upper byte lanes the exponent moves DOWN, which the high half of a multiply-add does).
+template <int BITS, int STRIDE = 4>
+__device__ __forceinline__ void pot_decode32_bf16(const uint32_t* rec, int T, uint32_t sc2, uint32_t (&out)[16]) {
+    using L = PotLanes<BITS>;
+    constexpr uint32_t EM = L::MASK & 0x7F7F7F7Fu, SM = L::MASK & 0x80808080u;
+    constexpr uint32_t LA = 0x00FF00FFu, LB = 0xFF00FF00u;
+    uint32_t w[BITS], d[8];
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) w[k] = rec[STRIDE * k + T];
+    L::rotate(w, d);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int p = L::low(i);
+        // lower byte lanes (columns 2p', 2p'+1 of the pair 2i): exponent from bit 2 - p up to bit 7, sign to bit 15
+        const uint32_t ea = mad(d[i] & ((EM & LA) >> p), 1u << (5 + p), sc2);
+        out[2 * i] = mad(d[i] & ((SM & LA) >> p), 1u << (8 + p), ea);
+        // upper byte lanes: exponent from bit 10 - p down to bit 7, sign from bit 15 - p up to bit 15
+        const uint32_t eb = madhi(d[i] & ((EM & LB) >> p), 1u << (29 + p), sc2);
+        out[2 * i + 1] = p == 0 ? (eb | (d[i] & (SM & LB))) : mad(d[i] & ((SM & LB) >> p), 1u << p, eb);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Uniform-INT twin on the same tiled layout: w~ = (q - z) * s with q spliced under the exponent
 // of 1024 (0x6400 | q = 1024 + q as FP16), an exact subtraction, and one rounding multiply.

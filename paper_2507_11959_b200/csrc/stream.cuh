@@ -116,8 +116,8 @@ struct StreamArgs {
     const unsigned char* packed;   // tiled codes
     const unsigned char* scales;   // tiled scales
     const unsigned char* zeros;    // tiled zero-points (uniform twin)
-    const __half* X;
-    __half* Y;
+    const uint16_t* X;             // FP16 or BF16 bit patterns
+    uint16_t* Y;
     float* partial;
     unsigned* counters;
     int64_t N, K;
@@ -138,6 +138,19 @@ __device__ __forceinline__ void sk_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void sk_mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                            uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// FP32 sum -> 16-bit output pattern (DT = 0: FP16, 1: BF16), round to nearest even
+template <int DT>
+__device__ __forceinline__ uint16_t sk_out(float v) {
+    if (DT == 0) return __half_as_ushort(__float2half_rn(v));
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
 __device__ __forceinline__ uint32_t sk_lds32(const unsigned char* p) { return *reinterpret_cast<const uint32_t*>(p); }
 __device__ __forceinline__ uint4 sk_lds128(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
 // floor(a * b / c) for a * b that may need 64 bits
@@ -146,11 +159,13 @@ __device__ __forceinline__ uint32_t sk_muldiv(uint32_t a, uint32_t b, uint32_t c
     return (uint32_t)(((uint64_t)a * (uint64_t)b) / (uint64_t)c);
 }
 
+// DT = 0: FP16 activations, weights and output; DT = 1: BF16 (PoT codes only: the scale is rounded once to BF16 and the
+// exponent is added at bit 7).
 // KIND: SK_POT / SK_UINT.  TOK = 1: GEMV (x in every B column).  TOK = 8: up to 8 tokens, one per B column.
 // XSMEM: the activations are staged in shared memory in fragment order (else they are read through L1 from global).
 // W consumer warps per CTA; OCC = 2 leaves room for a second CTA on the SM (64 registers per thread, half the shared
 // memory), so that the next launch in the stream can become resident and fill its rings while this one still computes.
-template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1, int SK_Q = SK_QMAX>
+template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1, int SK_Q = SK_QMAX, int DT = 0>
 __global__ void __launch_bounds__(W * 32, OCC)
 stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     constexpr int UB = sk_unit_bytes(BITS);
@@ -289,15 +304,15 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         if (expect == 0) {
             if constexpr (TOK == 1) {
                 if (tig == 0 && in_range(row0 + gid + 8 < sa.N, err, 0x120)) {
-                    sa.Y[row0 + gid] = __float2half_rn(v[0]);
-                    sa.Y[row0 + gid + 8] = __float2half_rn(v[2]);
+                    sa.Y[row0 + gid] = sk_out<DT>(v[0]);
+                    sa.Y[row0 + gid + 8] = sk_out<DT>(v[2]);
                 }
             } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int token = 2 * tig + (e & 1);
                     if (token < sa.M && in_range(row0 + gid + 8 * (e >> 1) < sa.N, err, 0x121))
-                        sa.Y[(int64_t)token * sa.N + row0 + gid + 8 * (e >> 1)] = __float2half_rn(v[e]);
+                        sa.Y[(int64_t)token * sa.N + row0 + gid + 8 * (e >> 1)] = sk_out<DT>(v[e]);
                 }
             }
             return;
@@ -326,7 +341,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
                 for (int e = lane; e < 16 * (TOK == 1 ? 1 : sa.M); e += 32) {
                     float sum = 0.f;
                     for (uint32_t q = 0; q < expect; ++q) sum += lslots[((size_t)(wl + q) * 2 + (q == 0 ? 1 : 0)) * (16 * TOK) + e];
-                    sa.Y[(int64_t)(e >> 4) * sa.N + row0 + (e & 15)] = __float2half_rn(sum);
+                    sa.Y[(int64_t)(e >> 4) * sa.N + row0 + (e & 15)] = sk_out<DT>(sum);
                 }
             }
             return;
@@ -358,7 +373,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             for (int e = lane; e < 16 * (TOK == 1 ? 1 : sa.M); e += 32) {
                 float sum = 0.f;
                 for (uint32_t q = 0; q < expect; ++q) sum += __ldcg(base + (size_t)q * (16 * TOK) + e);
-                sa.Y[(int64_t)(e >> 4) * sa.N + row0 + (e & 15)] = __float2half_rn(sum);
+                sa.Y[(int64_t)(e >> 4) * sa.N + row0 + (e & 15)] = sk_out<DT>(sum);
             }
             if (lane == 0) sa.counters[rbd] = 0u;  // leave the workspace ready for the next call
         }
@@ -402,8 +417,15 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
 #pragma unroll
                 for (int k = 0; k < BITS; ++k) w[h][k] = sk_lds32(code + (uint32_t)(k * 256 + h * 128) + (uint32_t)lane * 4u);
             const uint32_t scw = sk_lds32(param + poff);  // {row gid, row gid + 8}
-            potl::pot_decode32<BITS, 1>(w[0], 0, __byte_perm(scw, 0, 0x1010), lo);
-            potl::pot_decode32<BITS, 1>(w[1], 0, __byte_perm(scw, 0, 0x3232), hi);
+            if constexpr (DT == 0) {
+                potl::pot_decode32<BITS, 1>(w[0], 0, __byte_perm(scw, 0, 0x1010), lo);
+                potl::pot_decode32<BITS, 1>(w[1], 0, __byte_perm(scw, 0, 0x3232), hi);
+            } else {  // the FP16 scale rounded once to BF16
+                const uint32_t s0 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)(scw & 0xFFFFu)))));
+                const uint32_t s1 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)(scw >> 16)))));
+                potl::pot_decode32_bf16<BITS, 1>(w[0], 0, s0 * 0x10001u, lo);
+                potl::pot_decode32_bf16<BITS, 1>(w[1], 0, s1 * 0x10001u, hi);
+            }
         } else {
             // the quarter's words sit at record words 2 tig, 2 tig + 1 (n = 2), 2 tig, 2 tig + 1, 8 + tig (n = 3) or
             // 4 tig .. 4 tig + 3 (n = 4); record word w is byte (w / 4) * 256 + row * 16 + (w % 4) * 4
@@ -433,7 +455,8 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j)  // two accumulators: half the length of the dependent chain
-            sk_mma(acc[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
+            if constexpr (DT == 0) sk_mma(acc[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
+            else sk_mma_bf16(acc[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
     };
 
     // ---- main loop over this warp's chunks --------------------------------------------------------------------
@@ -494,8 +517,8 @@ inline StreamArgs stream_args(const StreamPlan& p, const void* packed, const voi
     sa.packed = (const unsigned char*)packed;
     sa.scales = (const unsigned char*)scales;
     sa.zeros = (const unsigned char*)zeros;
-    sa.X = (const __half*)X;
-    sa.Y = (__half*)Y;
+    sa.X = (const uint16_t*)X;
+    sa.Y = (uint16_t*)Y;
     sa.counters = (unsigned*)workspace;
     sa.partial = workspace ? (float*)((char*)workspace + p.ws_counters) : nullptr;
     sa.N = N;
@@ -519,7 +542,7 @@ inline StreamArgs stream_args(const StreamPlan& p, const void* packed, const voi
 }
 
 #ifdef __CUDACC__
-template <int BITS, int KIND, int TOK, int W, int OCC = 1>
+template <int BITS, int KIND, int TOK, int W, int OCC = 1, int DT = 0>
 pot_status_t launch_stream(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K, int group,
                            const void* X, int M, void* Y, void* workspace, int* err, cudaStream_t s) {
     const StreamPlan p = plan_stream(N, K, M, BITS, group, KIND, TOK, W, OCC);
@@ -530,11 +553,11 @@ pot_status_t launch_stream(const void* packed, const void* scales, const void* z
         return launch_pdl(kernel, dim3((unsigned)p.grid), dim3(W * 32), p.smem_bytes, s, sa, err);
     };
     if (p.q == 2) {
-        if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2>);
-        return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2>);
+        if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2, DT>);
+        return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2, DT>);
     }
-    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, SK_QMAX>);
-    return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, SK_QMAX>);
+    if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, SK_QMAX, DT>);
+    return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, SK_QMAX, DT>);
 }
 #endif
 
