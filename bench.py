@@ -149,6 +149,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config tables (chain only)")
     ap.add_argument("--layers", type=int, default=synth.LLAMA2_7B_LAYERS)
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
+                    help="N > 1: 'replicas' = every rank runs the whole chain (weak scaling, the default); 'rows' = every "
+                         "projection is split by rows over the ranks and the outputs are all-gathered (strong scaling)")
     ap.add_argument("--kernel", default=None, choices=["gemv", "gemv_uint", "dequant", "dequant_uint", "gemm"],
                     help="profiling mode: run only this kernel on one small seeded case and print its timing")
     ap.add_argument("--N", type=int, default=12288)
@@ -240,6 +243,10 @@ def main():
             per_step.extend(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
         return ev[0].elapsed_time(ev[-1]) / steps  # ms per step
 
+    if args.shard == "rows":
+        sharded_rows_arm(args, B, pdist, torch, dev, stream, f16, peaks, rank, world)
+        return
+
     layers3, bytes3 = build_chain(HEADLINE_BITS)
     launches_before = B.pot_launch_count()
     g3 = capture(lambda s: enqueue_chain(layers3, HEADLINE_BITS, s))
@@ -326,6 +333,71 @@ def main():
     del layers3
     if rank == 0:
         print(json.dumps(out))
+
+
+def sharded_rows_arm(args, B, pdist, torch, dev, stream, f16, peaks, rank, world):
+    """The 7B chain with every projection split by rows over the ranks (RowShard) and an NCCL all-gather of y after each
+    GEMV: the whole job is ONE model, so the value is the model's bytes over the step time (strong scaling).  Eager
+    launches on one stream (the collective sits between the GEMVs)."""
+    protos, nbytes = [], 0
+    for i, pr in enumerate(synth.LLAMA2_7B):
+        W = f16(synth.weights(synth.rng_for(2, 2 * i), pr.N, pr.K, "t5"))
+        packed, S = B.pot_quantize_ref(W, HEADLINE_BITS, GROUP, B.SCALE_TOP)
+        sh = pdist.RowShard(packed, S, pr.K, HEADLINE_BITS, GROUP, rank, world)
+        x = f16(synth.activations(synth.rng_for(2, 2 * i + 1), 1, pr.K)[0])
+        y_full = torch.empty(pr.N, dtype=torch.float16, device=dev)
+        ws = B.new_workspace(B.pot_gemv_workspace_bytes(sh.end - sh.begin, pr.K, HEADLINE_BITS, GROUP), dev) if sh.end > sh.begin else None
+        protos.append((sh, x, y_full, ws))
+        nbytes += gemv_bytes(pr.N, pr.K, HEADLINE_BITS, GROUP)
+        del W, packed, S
+    layers = []
+    for _ in range(args.layers):  # distinct weight buffers per layer: the chain streams from HBM
+        layer = []
+        for sh, x, y_full, ws in protos:
+            c = pdist.RowShard.__new__(pdist.RowShard)
+            c.__dict__.update(sh.__dict__)
+            c.codes, c.scales = sh.codes.clone(), sh.scales.clone()
+            layer.append((c, x, y_full, ws))
+        layers.append(layer)
+    nbytes *= args.layers
+
+    def step():
+        for layer in layers:
+            for sh, x, y_full, ws in layer:
+                pdist.sharded_gemv(sh, x, y_full, workspace=ws, stream=stream)
+
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", 0)))
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
+        stream.synchronize()
+        pdist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        before = B.pot_launch_count()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        pdist.barrier()
+    clocks = sampler.stop()
+    ms = pdist.max_over_ranks(e0.elapsed_time(e1) / args.steps, dev)
+    value = nbytes / (ms * 1e-3) / 1e9
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f16 (int32 bit ops, f32 accumulate)", "data": "synthetic",
+            "config": {"workload": f"llama2-7b-shaped decode chain, batch 1, {args.layers} layers x 5 projections, PoT {HEADLINE_BITS}-bit g{GROUP}, "
+                                   f"rows of every projection sharded over {world} ranks, NCCL all-gather of y after every GEMV, eager launches",
+                       "l2": "inputs larger than L2", "bytes_per_step": nbytes},
+            "clocks": clocks, "gpu_launches": B.pot_launch_count() - before,
+            "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": value / world / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None},
+            "e2e": None, "cpu_baseline": None}))
 
 
 def single_kernel(args):
