@@ -38,6 +38,10 @@ template <int BITS, int EBIT>
 __global__ void __launch_bounds__(DQ_THREADS) pot_dequant_kernel(const uint32_t* __restrict__ packed,
                                                                  const uint16_t* __restrict__ scales, int64_t n_pieces,
                                                                  int ppg_shift, uint4* __restrict__ out) {
+    // programmatic dependent launch: this grid may have been scheduled while its predecessor in the stream was still
+    // running; nothing is read or written before the predecessor has completed
+    pdl_wait();
+    pdl_launch_dependents();
     constexpr uint32_t QM2 = (uint32_t)qmax_of(BITS) * 0x10001u;   // exponent mask, both halves
     constexpr uint32_t SM2 = (1u << (BITS - 1)) * 0x10001u;        // sign mask, both halves
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
@@ -85,6 +89,10 @@ template <int EBIT>
 __global__ void __launch_bounds__(DQ_THREADS) pot_dequant3_kernel(const uint32_t* __restrict__ packed,
                                                                   const uint16_t* __restrict__ scales, int64_t n_pieces,
                                                                   int ppg_shift, uint4* __restrict__ out) {
+    // programmatic dependent launch: this grid may have been scheduled while its predecessor in the stream was still
+    // running; nothing is read or written before the predecessor has completed
+    pdl_wait();
+    pdl_launch_dependents();
     constexpr uint32_t QM2 = (uint32_t)qmax_of(3) * 0x10001u, SM2 = 4u * 0x10001u;
     __shared__ uint4 tile[4 * DQ_THREADS];
     const int t = threadIdx.x;
@@ -127,6 +135,10 @@ __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_fast_kernel(const uin
                                                                        const uint16_t* __restrict__ zeros,
                                                                        int64_t n_pieces, int ppg_shift,
                                                                        uint4* __restrict__ out) {
+    // programmatic dependent launch: this grid may have been scheduled while its predecessor in the stream was still
+    // running; nothing is read or written before the predecessor has completed
+    pdl_wait();
+    pdl_launch_dependents();
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
     const int64_t bit0 = base * (8 * BITS);
     const uint32_t* w0 = packed + (bit0 >> 5);
@@ -168,6 +180,10 @@ __global__ void __launch_bounds__(DQ_THREADS) uint_dequant3_fast_kernel(const ui
                                                                         const uint16_t* __restrict__ scales,
                                                                         const uint16_t* __restrict__ zeros, int64_t n_pieces,
                                                                         int ppg_shift, uint4* __restrict__ out) {
+    // programmatic dependent launch: this grid may have been scheduled while its predecessor in the stream was still
+    // running; nothing is read or written before the predecessor has completed
+    pdl_wait();
+    pdl_launch_dependents();
     __shared__ uint4 tile[4 * DQ_THREADS];
     const int t = threadIdx.x;
     const int64_t base = (int64_t)blockIdx.x * (4 * DQ_THREADS);
@@ -208,6 +224,10 @@ __global__ void __launch_bounds__(DQ_THREADS) uint_dequant_naive_kernel(const ui
                                                                         const uint16_t* __restrict__ zeros,
                                                                         int64_t n_pieces, int ppg_shift,
                                                                         uint4* __restrict__ out) {
+    // programmatic dependent launch: this grid may have been scheduled while its predecessor in the stream was still
+    // running; nothing is read or written before the predecessor has completed
+    pdl_wait();
+    pdl_launch_dependents();
     constexpr uint32_t CM = (1u << BITS) - 1u;
     const int64_t base = ((int64_t)blockIdx.x * DQ_UNROLL) * DQ_THREADS + threadIdx.x;
 #pragma unroll
@@ -247,19 +267,20 @@ extern "C" pot_status_t pot_dequant(const void* packed, const void* scales, int6
     auto* S = (const uint16_t*)scales;
     auto* O = (uint4*)W_out;
     const int ppg = group == 64 ? 3 : 4;  // log2(pieces per group): a 64-bit division per piece would dominate the kernel
+    pot_status_t rc = POT_OK;
 #define POT_DQ(B)                                                                                     \
-    if (out_dtype == POT_F16) pot_dequant_kernel<B, 10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O); \
-    else pot_dequant_kernel<B, 7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
+    if (out_dtype == POT_F16) rc = launch_pdl(pot_dequant_kernel<B, 10>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, n_pieces, ppg, O); \
+    else rc = launch_pdl(pot_dequant_kernel<B, 7>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, n_pieces, ppg, O);
     if (bits == 2) {
         POT_DQ(2)
     } else if (bits == 3) {
-        if (out_dtype == POT_F16) pot_dequant3_kernel<10><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
-        else pot_dequant3_kernel<7><<<grid, DQ_THREADS, 0, s>>>(P, S, n_pieces, ppg, O);
+        if (out_dtype == POT_F16) rc = launch_pdl(pot_dequant3_kernel<10>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, n_pieces, ppg, O);
+        else rc = launch_pdl(pot_dequant3_kernel<7>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, n_pieces, ppg, O);
     } else {
         POT_DQ(4)
     }
 #undef POT_DQ
-    return launched();
+    return rc;
 }
 
 extern "C" pot_status_t uint_dequant(const void* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
@@ -277,17 +298,18 @@ extern "C" pot_status_t uint_dequant(const void* packed, const void* scales, con
     auto* Z = (const uint16_t*)zeros;
     auto* O = (uint4*)W_out;
     const int ppg = group == 64 ? 3 : 4;  // log2(pieces per group): a 64-bit division per piece would dominate the kernel
+    pot_status_t rc = POT_OK;
 #define UINT_DQ(B)                                                                                              \
-    if (kernel == UINT_KERNEL_FAST) uint_dequant_fast_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O); \
-    else uint_dequant_naive_kernel<B><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
+    if (kernel == UINT_KERNEL_FAST) rc = launch_pdl(uint_dequant_fast_kernel<B>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, Z, n_pieces, ppg, O); \
+    else rc = launch_pdl(uint_dequant_naive_kernel<B>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, Z, n_pieces, ppg, O);
     if (bits == 2) {
         UINT_DQ(2)
     } else if (bits == 3) {
-        if (kernel == UINT_KERNEL_FAST) uint_dequant3_fast_kernel<<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
-        else uint_dequant_naive_kernel<3><<<grid, DQ_THREADS, 0, s>>>(P, S, Z, n_pieces, ppg, O);
+        if (kernel == UINT_KERNEL_FAST) rc = launch_pdl(uint_dequant3_fast_kernel, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, Z, n_pieces, ppg, O);
+        else rc = launch_pdl(uint_dequant_naive_kernel<3>, dim3(grid), dim3(DQ_THREADS), 0, s, P, S, Z, n_pieces, ppg, O);
     } else {
         UINT_DQ(4)
     }
 #undef UINT_DQ
-    return launched();
+    return rc;
 }
