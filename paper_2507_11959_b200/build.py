@@ -49,7 +49,8 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
 
     def compile_one(src: str) -> Path:
         obj = OBJ_DIR / (src + ".o")
-        cmd = [nvcc, *flags, "-c", str(CSRC / src), "-o", str(obj)]
+        extra = os.environ.get("POT_NVCC_FLAGS_" + src.split(".")[0].upper(), "").split()
+        cmd = [nvcc, *flags, *extra, "-c", str(CSRC / src), "-o", str(obj)]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if verbose or r.returncode != 0:
             sys.stderr.write(f"$ {' '.join(cmd)}\n{r.stdout}{r.stderr}\n")

@@ -39,9 +39,10 @@ __host__ __device__ constexpr int sk_unit_total_bytes(int bits, int group, int k
 }
 __host__ __device__ constexpr int sk_slot_bytes(int bits, int group, int kind, int q) { return q * sk_unit_total_bytes(bits, group, kind); }
 
-// shared-memory header of a CTA: W x 8 full barriers, W local arrival counters, W x 2 local partial-sum slots
+// shared-memory header of a CTA: W x 8 full barriers, W x 8 words of per-warp state, W local arrival counters, W x 2 local
+// partial-sum slots
 __host__ __device__ constexpr int sk_header_bytes(int warps, int tok) {
-    return (warps * 64 + warps * 4 + warps * 2 * 16 * tok * 4 + 127) / 128 * 128;
+    return (warps * 64 + warps * 32 + warps * 4 + warps * 2 * 16 * tok * 4 + 127) / 128 * 128;
 }
 
 struct StreamPlan {
@@ -165,9 +166,8 @@ __device__ __forceinline__ uint32_t sk_muldiv(uint32_t a, uint32_t b, uint32_t c
 // XSMEM: the activations are staged in shared memory in fragment order (else they are read through L1 from global).
 // W consumer warps per CTA; OCC = 2 leaves room for a second CTA on the SM (64 registers per thread, half the shared
 // memory), so that the next launch in the stream can become resident and fill its rings while this one still computes.
-template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1, int SK_Q = SK_QMAX, int DT = 0>
-__global__ void __launch_bounds__(W * 32, OCC)
-stream_kernel(const StreamArgs sa, int* __restrict__ err) {
+template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC, int SK_Q, int DT>
+__device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restrict__ err) {
     constexpr int UB = sk_unit_bytes(BITS);
     constexpr bool UNIFORM = (KIND == SK_UINT);
     constexpr int NPARAM = UNIFORM ? 2 : 1;
@@ -193,8 +193,13 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bars = smem0 + (uint32_t)warp * 64u;      // this warp's full barriers (S <= 8)
     constexpr int HDR = sk_header_bytes(W, TOK);
-    unsigned* lcnt = reinterpret_cast<unsigned*>(smem + W * 64);               // local arrival counters
-    float* lslots = reinterpret_cast<float*>(smem + W * 64 + W * 4);           // [warp][first, last][16 TOK]
+    // Values a warp needs only when it requests a chunk or delivers sums live in shared memory, not in registers (the
+    // two-CTAs-per-SM build has 64 registers per thread): [0] a, [1] n, [2] first row block, [3] last row block,
+    // [4] slot of the first segment, [5] contributors of the first segment, [6] of the last, [7] bit 0 / 1: the first / last
+    // segment is combined inside the CTA
+    uint32_t* wst = reinterpret_cast<uint32_t*>(smem + W * 64) + warp * 8;
+    unsigned* lcnt = reinterpret_cast<unsigned*>(smem + W * 96);               // local arrival counters
+    float* lslots = reinterpret_cast<float*>(smem + W * 96 + W * 4);           // [warp][first, last][16 TOK]
     const unsigned char* xs = smem + HDR;
     const unsigned char* ringp = xs + sa.x_bytes + (uint32_t)warp * (uint32_t)S * slot_bytes;  // this warp's ring
     const uint32_t ring = smem0 + (uint32_t)HDR + (uint32_t)sa.x_bytes + (uint32_t)warp * (uint32_t)S * slot_bytes;
@@ -217,23 +222,21 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     const uint32_t nchunks = (n + SK_Q - 1) / SK_Q;
 
     // chunk j of the range holds units [a + Q j, a + Q j + Q) (fewer at the end) and lives in slot j % S
-    const unsigned char* pk = sa.packed + (size_t)a * UB;
-    const unsigned char* ps = sa.scales + (size_t)a * PB;
-    const unsigned char* pz = UNIFORM ? sa.zeros + (size_t)a * PB : nullptr;
-    auto issue = [&](uint32_t j, uint32_t s) {  // lane 0: request chunk j into slot s
-        const uint32_t left_j = n - j * SK_Q;
+    auto issue = [&](uint32_t a_, uint32_t n_, uint32_t j, uint32_t s) {  // one lane: request chunk j into slot s
+        const uint32_t left_j = n_ - j * SK_Q;
         const uint32_t cnt = left_j < (uint32_t)SK_Q ? left_j : (uint32_t)SK_Q;
         const uint32_t bar = bars + s * 8u, dst = ring + s * slot_bytes;
-        if (!in_range(s < (uint32_t)S && a + j * SK_Q + cnt <= sa.units && cnt >= 1, err, 0x110)) return;
+        const size_t u0 = (size_t)a_ + (size_t)j * SK_Q;
+        if (!in_range(s < (uint32_t)S && u0 + cnt <= sa.units && cnt >= 1 && cnt <= (uint32_t)SK_Q, err, 0x110)) return;
         mbar_expect_tx(bar, cnt * (UB + NPARAM * PB));
-        bulk_g2s(dst, pk + (size_t)j * (SK_Q * UB), cnt * UB, bar);
-        bulk_g2s(dst + SK_Q * UB, ps + (size_t)j * SK_Q * PB, cnt * PB, bar);
-        if constexpr (UNIFORM) bulk_g2s(dst + SK_Q * (UB + PB), pz + (size_t)j * SK_Q * PB, cnt * PB, bar);
+        bulk_g2s(dst, sa.packed + u0 * UB, cnt * UB, bar);
+        bulk_g2s(dst + SK_Q * UB, sa.scales + u0 * PB, cnt * PB, bar);
+        if constexpr (UNIFORM) bulk_g2s(dst + SK_Q * (UB + PB), sa.zeros + u0 * PB, cnt * PB, bar);
     };
     if (lane < S) {  // lane s sets up slot s and requests chunk s: the weights do not depend on the predecessor
         mbar_init(bars + (uint32_t)lane * 8u, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if ((uint32_t)lane < nchunks) issue((uint32_t)lane, (uint32_t)lane);
+        if ((uint32_t)lane < nchunks) issue(a, n, (uint32_t)lane, (uint32_t)lane);
     }
     __syncwarp();
     stamp(7);
@@ -260,6 +263,10 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     const uint32_t cta_lo = sa.aligned ? 0u : blockIdx.x * W;
     const bool loc0 = exp0 && gw - slot0 >= cta_lo && gw - slot0 + exp0 <= cta_lo + W;
     const bool locL = expL && gw + expL <= cta_lo + W;
+    if (lane == 0) {
+        wst[0] = a; wst[1] = n; wst[2] = rb0; wst[3] = rbL;
+        wst[4] = slot0; wst[5] = exp0; wst[6] = expL; wst[7] = (loc0 ? 1u : 0u) | (locL ? 2u : 0u);
+    }
     if (threadIdx.x < W) lcnt[threadIdx.x] = 0u;
 
     stamp(1);
@@ -298,8 +305,9 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             acc[0][e] = 0.f;
             acc[1][e] = 0.f;
         }
-        const uint32_t expect = rbd == rb0 ? exp0 : (rbd == rbL ? expL : 0u);
-        const uint32_t slot = rbd == rb0 ? slot0 : 0u;
+        const bool first = rbd == wst[2];
+        const uint32_t expect = first ? wst[5] : (rbd == wst[3] ? wst[6] : 0u);
+        const uint32_t slot = first ? wst[4] : 0u;
         const int64_t row0 = (int64_t)rbd * 16;
         if (expect == 0) {
             if constexpr (TOK == 1) {
@@ -317,7 +325,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             }
             return;
         }
-        if (rbd == rb0 ? loc0 : locL) {
+        if ((wst[7] >> (first ? 0 : 1)) & 1u) {
             // slot of warp w: [w][1] if w is the row block's first contributor, else [w][0]
             const uint32_t wl = (uint32_t)warp - slot;  // first contributor (local warp index)
             if (!in_range(slot <= (uint32_t)warp && wl + expect <= (uint32_t)W && row0 + 16 <= sa.N, err, 0x130)) return;
@@ -461,7 +469,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
 
     // ---- main loop over this warp's chunks --------------------------------------------------------------------
     uint32_t s = 0, phase = 0, left = n;
-    for (uint32_t j = 0; j < nchunks; ++j) {
+    for (uint32_t j = 0; left > 0; ++j) {
         const unsigned char* code = ringp + s * slot_bytes;
         const unsigned char* param = code + SK_Q * UB;
         const uint32_t bar = bars + s * 8u;
@@ -495,7 +503,7 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
             left -= cnt;
         }
         __syncwarp();  // every lane has read the slot: it may be refilled
-        if (lane == 0 && j + (uint32_t)S < nchunks) issue(j + (uint32_t)S, s);
+        if (lane == 0 && (j + (uint32_t)S) * SK_Q < wst[1]) issue(wst[0], wst[1], j + (uint32_t)S, s);
         if (++s == (uint32_t)S) {
             s = 0;
             phase ^= 1u;
@@ -504,6 +512,11 @@ stream_kernel(const StreamArgs sa, int* __restrict__ err) {
     stamp(5);
     if (n && cb != 0) deliver(rb);
     stamp(6);
+}
+
+template <int BITS, int KIND, int TOK, bool XSMEM, int W, int OCC = 1, int SK_Q = SK_QMAX, int DT = 0>
+__global__ void __launch_bounds__(W * 32, OCC) stream_kernel(const StreamArgs sa, int* __restrict__ err) {
+    stream_body<BITS, KIND, TOK, XSMEM, W, OCC, SK_Q, DT>(sa, err);
 }
 #endif  // __CUDACC__
 
