@@ -474,7 +474,18 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         const unsigned char* param = code + SK_Q * UB;
         const uint32_t bar = bars + s * 8u;
         if (!mbar_test(bar, phase) && !mbar_wait(bar, phase)) {
+            // A copy never arrived.  Record it, request nothing more, deliver nothing more (the rows this warp still owed
+            // stay unwritten: the error word says so), wait -- bounded again -- for the chunks already requested, leave.
             if (err && lane == 0) atomicCAS(err, 0, 2 | (int)(j << 8) | (warp << 24));
+            uint32_t s2 = s, ph2 = phase;
+            for (uint32_t k = 1; k < (uint32_t)S && (j + k) * SK_Q < wst[1]; ++k) {
+                if (++s2 == (uint32_t)S) {
+                    s2 = 0;
+                    ph2 ^= 1u;
+                }
+                mbar_wait(bars + s2 * 8u, ph2);
+            }
+            return;
         }
         if (j == 0) stamp(4);
         if (left >= (uint32_t)SK_Q && cb + (uint32_t)SK_Q <= ncb) {
