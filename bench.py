@@ -265,7 +265,7 @@ def main():
     # call (H2D of x, kernel, D2H of y on the call's stream); the calls go round-robin to E2E_LANES streams, each with
     # its own device and host buffers, so that one call's copies overlap another call's kernel -- the way a server
     # pipelines independent requests.  The captured graph holds the lanes as parallel branches.
-    E2E_LANES = 4
+    E2E_LANES = 8  # measured: 2 lanes 2.36 ms, 4 lanes 1.41 ms, 8 lanes 1.10 ms, 16 lanes 1.41 ms per step
     lane_streams = [torch.cuda.Stream(device=dev) for _ in range(E2E_LANES)]
     lane_bufs = []
     for _ in range(E2E_LANES):
@@ -305,7 +305,7 @@ def main():
     h2d = args.layers * sum(2 * pr.K for pr in synth.LLAMA2_7B)
     d2h = args.layers * sum(2 * pr.N for pr in synth.LLAMA2_7B)
     e2e = {"value": world * bytes3 / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "ms_per_step": ms_e2e, "results_checked_against_device_chain": True, "note": "x from pinned host and y to pinned host for each of the 160 GEMVs (pot_gemv_host), calls spread over 4 streams; weights resident in HBM"}
+           "ms_per_step": ms_e2e, "results_checked_against_device_chain": True, "note": "x from pinned host and y to pinned host for each of the 160 GEMVs (pot_gemv_host), calls spread over 8 streams; weights resident in HBM"}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
