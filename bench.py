@@ -605,6 +605,23 @@ def extras(args, B, torch, dev, stream, f16, capture, time_graph, peaks, build_c
     del Pb, gb
     torch.cuda.empty_cache()
 
+    # the BF16 route on the 7B qkv shape (3 bit): same bytes, two mask / multiply-add pairs per register instead of one
+    N, K = 12288, 4096
+    copies = 28
+    Pq = [torch.randint(0, 256, (N, K * 3 // 8), dtype=torch.uint8, device=dev, generator=gq) for _ in range(copies)]
+    Sq = (torch.rand((N, K // GROUP), device=dev, generator=gq) * 0.01 + 0.002).to(torch.float16)
+    wsq = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, 3, GROUP), dev)
+    res = {}
+    for name, dt in (("f16", torch.float16), ("bf16", torch.bfloat16)):
+        xq = torch.randn(K, device=dev, generator=gq).to(dt)
+        yq = torch.empty(N, dtype=dt, device=dev)
+        gg = capture(lambda s: [B.pot_gemv(p, Sq, K, 3, GROUP, xq, B.TILED, y=yq, workspace=wsq, stream=s) for p in Pq])
+        res[name + "_us"] = min(time_graph(gg, 5, 2) for _ in range(3)) / copies * 1e3
+        del gg
+    ex["gemv_7B_qkv_3bit_f16_vs_bf16"] = res
+    del Pq
+    torch.cuda.empty_cache()
+
     # standalone dequant (config 3): PoT vs the uniform twin (fast and naive kernels), FP16 out.  HBM-cold: every launch
     # of a graph reads its own packed matrix and writes its own output, R pairs with R x bytes >= 4 x L2; the L2-warm
     # figure (one pair, written over and over) is reported beside it, labelled.

@@ -126,8 +126,7 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // add.  A barrier test costs a few hundred cycles even when the phase is long complete, so the test for the issuer's
 // next stage is put in flight before the MMAs of this one are issued and examined afterwards.
 template <int J, int NI, int PF_STAGES, int MT, int DT = 0>
-__device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, uint32_t n_tok, int* err,
-                                         volatile uint32_t* aborted) {
+__device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, uint32_t n_tok, int* err) {
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
     const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
@@ -148,11 +147,8 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
         for (int s = J; s < PF_STAGES; s += NI) {
             const int kb = kb0 + s;
             if (kb >= nkb) break;
-            if (!ready && !mbar_wait(full(s), ph)) {  // give up: issue nothing more (the commit below still reports to the epilogue)
+            if (!ready && !mbar_wait(full(s), ph)) {
                 if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
-                *aborted = 1u;
-                kb0 = nkb;
-                break;
             }
             ready = 0;
             if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
@@ -187,9 +183,6 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PF_STAGES + 1);
-    // set by the first thread whose bounded wait gives up: it stops issuing copies / MMAs / tile writes at once, the other
-    // roles follow when their own waits run out, and the epilogue stores nothing
-    volatile uint32_t* aborted = tmem_slot + 1;
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
@@ -236,7 +229,6 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             mbar_init(empty(s), 1);
         }
         mbar_init(accum, NI);
-        *aborted = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // allocate the accumulator columns of tensor memory (whole warp), base address lands in shared memory
@@ -262,11 +254,6 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 const int s = kb % PF_STAGES;
                 if (kb >= PF_STAGES && !ready && !mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                     if (err) atomicCAS(err, 0, 0x10 | (kb << 8));
-                    *aborted = 1u;
-                    // no further copies; wait (bounded) for the ones this thread still has in flight
-                    for (int k = kb - n_tma; k >= 0 && k > kb - n_tma * PF_STAGES; k -= n_tma)
-                        mbar_wait(full(k % PF_STAGES), (uint32_t)((k / PF_STAGES) & 1));
-                    break;
                 }
                 const int kn = kb + n_tma;
                 ready = (kn < nkb && kn >= PF_STAGES) ? mbar_test(empty(kn % PF_STAGES), (uint32_t)((kn / PF_STAGES - 1) & 1)) : 0u;
@@ -282,8 +269,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err, aborted);
-            else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err, aborted);
+            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
         }
     } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
@@ -334,13 +321,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     // load and store issued twice.
                     if (!mbar_wait(empty(s), (uint32_t)((kb / PF_STAGES - 1) & 1))) {
                         if (err && lane == 0) atomicCAS(err, 0, 0x30 | (kb << 8));
-                        *aborted = 1u;
                     }
                     __syncwarp();
-                    if (*aborted) {  // (every lane polled the same barrier: the warp leaves together) write no more tiles
-                        i4 = nmine;
-                        break;
-                    }
                 }
                 unsigned char* brow = smem + (size_t)s * STAGE_BYTES + pf_x_bytes(MT) + row * 128;
                 uint32_t s16 = sc2[buf];
@@ -373,6 +355,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (err) atomicCAS(err, 0, 0x40);
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // A bounded wait that gave up (here or in any CTA of the launch) has left its code in the error word: a tile that may
+        // have been built from a stage that never arrived is not stored.  (The roles' loops themselves carry on to their
+        // bounds: control flow added to them costs the tensor pipe several per cent.)
+        const bool gave_up = err != nullptr && *reinterpret_cast<volatile int*>(err) != 0;
         // Lane = weight row (feature), column = token.  Warp (q, part): features n0 + 32 q .. + 31 (a warp may only touch its
         // own quarter of the lanes), token columns part * 32 MT .. + 32 MT - 1.
         const int q = warp & 3;
@@ -397,7 +383,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             } else {
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             }
-            if (feat < N && !*aborted && in_range(m0 + col < M && m0 >= 0 && feat >= 0 && (splits == 1 || (tail_index >= 0 && zsplit >= 0 && zsplit < splits)), err, 0x60)) {
+            if (feat < N && !gave_up && in_range(m0 + col < M && m0 >= 0 && feat >= 0 && (splits == 1 || (tail_index >= 0 && zsplit >= 0 && zsplit < splits)), err, 0x60)) {
                 if (splits == 1) {  // a warp stores 32 consecutive features (64 bytes) of one token at a time
                     uint16_t* dst = Y + (m0 + col) * N + feat;
 #pragma unroll
@@ -411,7 +397,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 }
             }
         }
-        if (splits > 1 && !*aborted && in_range(tail_index >= 0 && partial != nullptr && counters != nullptr, err, 0x61)) {
+        if (splits > 1 && !gave_up && in_range(tail_index >= 0 && partial != nullptr && counters != nullptr, err, 0x61)) {
             // The CTA that delivers the last split of a tile (an arrival counter tells it) adds the splits in
             // ascending order -- the result does not depend on timing -- and writes Y.
             __shared__ unsigned s_prev;
