@@ -98,9 +98,10 @@ uint64_t pot_launch_count(void);
 int pot_debug_gemv_error(void);
 /* Host arithmetic only: the launch plan pot_gemv (uniform = 0) / uint_gemv (uniform = 1) would use for a tiled shape:
  * CTAs per SM (1 or 2), whether CTA ranges end on row-block boundaries (1) or the units are split evenly and partial
- * sums cross CTAs through the workspace (0), slots per warp ring, and whether x is staged in shared memory.        */
+ * sums cross CTAs through the workspace (0), slots per warp ring, units per slot (2, 4 or 8), and whether x is staged
+ * in shared memory.                                                                                                  */
 pot_status_t pot_debug_gemv_plan(int64_t N, int64_t K, int bits, int group, int uniform, int* ctas_per_sm,
-                                 int* row_block_split, int* ring_slots, int* x_in_smem);
+                                 int* row_block_split, int* ring_slots, int* units_per_slot, int* x_in_smem);
 int pot_debug_gemm_error(void);
 int pot_debug_prefill_error(void);
 

@@ -62,7 +62,7 @@ def lib() -> ctypes.CDLL:
         L.pot_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.uint_repack.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.pot_repack_scales.argtypes = [vp, vp, i64, i64, i32, i32, vp]
-        L.pot_debug_gemv_plan.argtypes = [i64, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.pot_debug_gemv_plan.argtypes = [i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
         L.pot_layout_scale_index.argtypes = [i64, i64, i32, i64, i64, vp]
         L.pot_dequant.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.pot_gemv.argtypes = [vp, vp, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
@@ -291,10 +291,10 @@ def pot_gemv_noalloc(packed_tiled, scales, K: int, bits: int, group: int, x: tor
 
 
 def pot_debug_gemv_plan(N: int, K: int, bits: int, group: int, uniform: bool = False) -> dict:
-    """{'ctas_per_sm', 'row_block_split', 'ring_slots', 'x_in_smem'} of the tiled GEMV launch for this shape."""
-    v = [ctypes.c_int(-1) for _ in range(4)]
+    """{'ctas_per_sm', 'row_block_split', 'ring_slots', 'units_per_slot', 'x_in_smem'} of the tiled GEMV launch."""
+    v = [ctypes.c_int(-1) for _ in range(5)]
     _check(lib().pot_debug_gemv_plan(N, K, bits, group, 1 if uniform else 0, *[ctypes.byref(x) for x in v]), "pot_debug_gemv_plan")
-    return dict(zip(("ctas_per_sm", "row_block_split", "ring_slots", "x_in_smem"), (x.value for x in v)))
+    return dict(zip(("ctas_per_sm", "row_block_split", "ring_slots", "units_per_slot", "x_in_smem"), (x.value for x in v)))
 
 
 def pot_debug_errors() -> tuple[int, int, int]:

@@ -131,8 +131,8 @@ using namespace pot;
 
 // Host arithmetic only: how pot_gemv / uint_gemv would run a tiled shape (tests assert which variants they reach).
 extern "C" pot_status_t pot_debug_gemv_plan(int64_t N, int64_t K, int bits, int group, int uniform, int* ctas_per_sm,
-                                            int* row_block_split, int* ring_slots, int* x_in_smem) {
-    if (!ctas_per_sm || !row_block_split || !ring_slots || !x_in_smem) return POT_ERR_NULL;
+                                            int* row_block_split, int* ring_slots, int* units_per_slot, int* x_in_smem) {
+    if (!ctas_per_sm || !row_block_split || !ring_slots || !units_per_slot || !x_in_smem) return POT_ERR_NULL;
     pot_status_t st = check_shape(N, K, bits, group);
     if (st != POT_OK) return st;
     if (N % 16 != 0) return POT_ERR_SHAPE;
@@ -143,6 +143,7 @@ extern "C" pot_status_t pot_debug_gemv_plan(int64_t N, int64_t K, int bits, int 
     *ctas_per_sm = occ;
     *row_block_split = p.aligned ? 1 : 0;
     *ring_slots = p.stages;
+    *units_per_slot = p.q;
     *x_in_smem = p.x_in_smem ? 1 : 0;
     return POT_OK;
 }

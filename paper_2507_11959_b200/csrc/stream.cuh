@@ -29,7 +29,7 @@ namespace pot {
 
 enum StreamKind { SK_POT = 0, SK_UINT = 1 };
 
-constexpr int SK_QMAX = 4;  // units per chunk (one ring slot, one set of bulk copies): 4, or 2 where 4 would leave one slot
+constexpr int SK_QMAX = 4;  // units per chunk (one ring slot, one set of bulk copies): 4; 2 where 4 would leave one slot; 8 for long ranges
 
 __host__ __device__ constexpr int sk_unit_bytes(int bits) { return 256 * bits; }
 // bytes of one ring slot: Q units of codes, then their scales (then their zero-points)
@@ -91,6 +91,8 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     // slots of 4 units unless the ring could then hold only one of them next to the staged activations
     int q = SK_QMAX;
     if (hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget) q = 2;
+    // long ranges (large matrices, one CTA per SM): slots of 8 units halve the per-slot hand-off work, if two of them fit
+    else if (occ == 1 && tok == 1 && per_warp >= 32 && hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, 8) <= budget) q = 8;
     p.q = q;
     const size_t slot = (size_t)sk_slot_bytes(bits, group, kind, q);
     const size_t ring2 = (size_t)warps * 2 * slot;  // at least two slots per warp
@@ -579,6 +581,9 @@ pot_status_t launch_stream(const void* packed, const void* scales, const void* z
     if (p.q == 2) {
         if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2, DT>);
         return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2, DT>);
+    }
+    if constexpr (OCC == 1 && TOK == 1) {
+        if (p.q == 8) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 8, DT>);  // only chosen with x in shared memory
     }
     if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, SK_QMAX, DT>);
     return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, SK_QMAX, DT>);

@@ -54,6 +54,7 @@ def test_config2_llama7b_projections(B, oracle, bits):
             continue  # same shape as gate
         plan = check_gemv(B, oracle, pr.N, pr.K, bits, "t5", (2, 2 * i))
         seen.add(plan["ctas_per_sm"])
+        assert plan["units_per_slot"] == (2 if pr.K == 11008 and bits == 3 else 4), (pr.name, plan)
     assert seen == {2}, seen
 
 
@@ -123,7 +124,8 @@ def test_config3_dequant_largest_matrix_sampled_rows(B, oracle, bits):
         assert np.array_equal(got, ref), (bits, dtype)
         del out
     # the same matrix through the fused GEMV (a share per CTA large enough for the one-CTA-per-SM variant)
-    assert B.pot_debug_gemv_plan(N, K, bits, G)["ctas_per_sm"] == 1
+    plan = B.pot_debug_gemv_plan(N, K, bits, G)
+    assert plan["ctas_per_sm"] == 1 and plan["units_per_slot"] == (4 if bits == 4 else 8), plan
     X = synth.activations(synth.rng_for(3, 650 + bits), 1, K)
     Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X, rows=rows)
     y = bits_of(B.pot_gemv(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X[0]), B.TILED))
