@@ -106,6 +106,15 @@ __device__ __forceinline__ bool in_range(bool, int*, int) { return true; }
 #endif
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// 16-byte load of data that the previous kernel in the stream may have written (activations, mostly).  Such data is
+// NOT read-only for the lifetime of a kernel that was launched early, so it must never go through the non-coherent
+// path (__ldg / ld.global.nc): the compiler may move those loads ahead of griddepcontrol.wait, and a load that was
+// moved returned the previous content of the buffer.  This one stays where it is written and reads through L2.
+__device__ __forceinline__ uint4 ld_dependent16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 

@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(128) pot_gemm_fallback_kernel(const uint32_t* 
         for (int idx = threadIdx.x; idx < 64 * 16; idx += 128) {
             const int r = idx >> 4, pc = idx & 15;
             uint4 xv = make_uint4(0, 0, 0, 0);
-            if (m0 + r < M) xv = __ldg(reinterpret_cast<const uint4*>(X + (m0 + r) * K + kb * 128) + pc);
+            if (m0 + r < M) xv = ld_dependent16(reinterpret_cast<const uint4*>(X + (m0 + r) * K + kb * 128) + pc);
             *reinterpret_cast<uint4*>(&Xs[r * FB_LD + pc * 8]) = xv;
             uint4 wv = make_uint4(0, 0, 0, 0);
             const int64_t row = n0 + r;

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(256) gemv_canonical_kernel(const uint32_t* __r
         const uint32_t v = read_bits(rowp, c * (8 * BITS), 8 * BITS);
         uint32_t s16 = __ldg(srow + (c * 8) / G);
         if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
-        const uint4 xv = __ldg(x + c);
+        const uint4 xv = ld_dependent16(x + c);
         const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {

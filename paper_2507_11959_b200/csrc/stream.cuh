@@ -280,13 +280,36 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         const int kc = (int)(sa.K / 8);  // 16-byte chunks per token
         if constexpr (TOK == 1) {
             // chunk (quarter t, part j) of a unit goes to position j * 4 + t: lanes tig = 0..3 read 64 contiguous bytes
-            for (int i = threadIdx.x; i < kc; i += W * 32) dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = __ldg(src + i);
+            // (four loads in flight per thread before the first store: one round trip for K <= 32 * 32 W)
+            for (int i0 = threadIdx.x; i0 < kc; i0 += 4 * W * 32) {
+                uint4 v[4];
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    if (i0 + p * W * 32 < kc) v[p] = ld_dependent16(src + i0 + p * W * 32);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const int i = i0 + p * W * 32;
+                    if (i < kc) dst[(i & ~15) | ((i & 3) << 2) | ((i >> 2) & 3)] = v[p];
+                }
+            }
         } else {
             // chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * 8 + token: a warp reads 512
             // contiguous bytes.  Tokens >= M stay unwritten: their columns of the product are never delivered.
-            for (int token = 0; token < sa.M; ++token)
-                for (int i = threadIdx.x; i < kc; i += W * 32)
-                    dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << 3) + token] = __ldg(src + (int64_t)token * kc + i);
+            const int total = sa.M * kc;  // X is [M][K]: chunk e belongs to token e / kc
+            for (int e0 = threadIdx.x; e0 < total; e0 += 4 * W * 32) {
+                uint4 v[4];
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    if (e0 + p * W * 32 < total) v[p] = ld_dependent16(src + e0 + p * W * 32);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const int e = e0 + p * W * 32;
+                    if (e < total) {
+                        const int token = e / kc, i = e - token * kc;
+                        dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << 3) + token] = v[p];
+                    }
+                }
+            }
         }
     }
     __syncthreads();
@@ -389,36 +412,15 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         }
     };
 
-    // ---- one unit: 2 x 32 codes of this lane -> 32 half2 -> eight MMAs ----------------------------------------
-    auto unit = [&](const unsigned char* code, const unsigned char* param, uint32_t cbu) {
-        if (!in_range(code >= ringp && code + UB <= ringp + (size_t)S * slot_bytes && param + NPARAM * PB <= ringp + (size_t)S * slot_bytes &&
-                          cbu < ncb && (!XSMEM || (size_t)(cbu + 1) * 256u * (TOK == 1 ? 1 : 8) <= (size_t)sa.x_bytes),
-                      err, 0x150))
-            return;
-        // activations of quarter tig (of token gid): the B fragments of the eight MMAs
-        uint32_t xq[16];
-        if constexpr (XSMEM) {
-            const unsigned char* xa = TOK == 1 ? xs + cbu * 256u + (uint32_t)tig * 16u
-                                               : xs + ((cbu * 16u + (uint32_t)tig) * 8u + (uint32_t)gid) * 16u;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 v = sk_lds128(xa + (TOK == 1 ? 64u : 512u) * i);
-                xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
-            }
-        } else {
-            const bool live = TOK == 1 || gid < sa.M;
-            const uint4* xp = reinterpret_cast<const uint4*>(sa.X) + (TOK == 1 || !live ? 0 : (int64_t)gid * (sa.K / 8)) +
-                              (int64_t)cbu * 16 + tig * 4;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (live) v = __ldg(xp + i);
-                xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
-            }
-        }
+    // ---- one unit: 2 x 32 codes of this lane -> 32 half2 (decode: needs no activations) -> eight MMAs (multiply) ----
+    auto unit_ok = [&](const unsigned char* code, const unsigned char* param, uint32_t cbu) {
+        return in_range(code >= ringp && code + UB <= ringp + (size_t)S * slot_bytes && param + NPARAM * PB <= ringp + (size_t)S * slot_bytes &&
+                            cbu < ncb && (!XSMEM || (size_t)(cbu + 1) * 256u * (TOK == 1 ? 1 : 8) <= (size_t)sa.x_bytes),
+                        err, 0x150);
+    };
+    auto decode = [&](const unsigned char* code, const unsigned char* param, uint32_t (&lo)[16], uint32_t (&hi)[16]) {
         // the scale words {row gid, row gid + 8} of this lane's group
         const uint32_t poff = ((spg == 2 ? (uint32_t)(tig >> 1) * 8u : 0u) + (uint32_t)gid) * 4u;
-        uint32_t lo[16], hi[16];
         if constexpr (!UNIFORM) {
             // plane k of a unit holds word k of every (row, quarter): this lane's word sits at byte 4 * lane
             uint32_t w[2][BITS];
@@ -463,10 +465,39 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
                 }
             }
         }
+    };
+    auto multiply = [&](const uint32_t (&lo)[16], const uint32_t (&hi)[16], uint32_t cbu) {
+        // activations of quarter tig (of token gid): the B fragments of the eight MMAs
+        uint32_t xq[16];
+        if constexpr (XSMEM) {
+            const unsigned char* xa = TOK == 1 ? xs + cbu * 256u + (uint32_t)tig * 16u
+                                               : xs + ((cbu * 16u + (uint32_t)tig) * 8u + (uint32_t)gid) * 16u;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = sk_lds128(xa + (TOK == 1 ? 64u : 512u) * i);
+                xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
+            }
+        } else {
+            const bool live = TOK == 1 || gid < sa.M;
+            const uint4* xp = reinterpret_cast<const uint4*>(sa.X) + (TOK == 1 || !live ? 0 : (int64_t)gid * (sa.K / 8)) +
+                              (int64_t)cbu * 16 + tig * 4;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (live) v = ld_dependent16(xp + i);
+                xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
+            }
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j)  // two accumulators: half the length of the dependent chain
             if constexpr (DT == 0) sk_mma(acc[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
             else sk_mma_bf16(acc[j & 1], lo[2 * j], hi[2 * j], lo[2 * j + 1], hi[2 * j + 1], xq[2 * j], xq[2 * j + 1]);
+    };
+    auto unit = [&](const unsigned char* code, const unsigned char* param, uint32_t cbu) {
+        if (!unit_ok(code, param, cbu)) return;
+        uint32_t lo[16], hi[16];
+        decode(code, param, lo, hi);
+        multiply(lo, hi, cbu);
     };
 
     // ---- main loop over this warp's chunks --------------------------------------------------------------------
