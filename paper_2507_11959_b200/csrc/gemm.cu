@@ -1,6 +1,7 @@
 // pot_gemm: Y[M,N] = X[M,K] W~^T with the dequantization fused in.
 //
-//  * M <= 8, tiled layout: the streaming tensor-core kernel of stream.cuh.  The weights are the MMA's
+//  * M = 1, tiled layout: the GEMV kernel (gemv.cu).
+//  * 2 <= M <= 8, tiled layout: the streaming tensor-core kernel of stream.cuh.  The weights are the MMA's
 //    M-side operand (16 rows per warp-step), the tokens its 8-wide N side, so no padding of M
 //    to 16 is needed and a warp decodes each record exactly once, straight into the A
 //    fragment registers -- the FP16 weights never exist in shared or global memory.
@@ -118,6 +119,8 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s, int dt);
 size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int bits, int group);
 bool gemm_prefill_supported(int64_t M, int64_t N, int64_t K, int bits, int group);
+pot_status_t gemv_stream_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group, const void* x,
+                                void* y, void* workspace, cudaStream_t s, int dt);
 
 }  // namespace pot
 
@@ -127,14 +130,24 @@ using namespace pot;
 // the tcgen05 kernel's time is flat in the batch but its floor is higher.  Measured on the 13B shapes: 13 - 23 us for
 // 1 - 8 tokens on the streaming kernel, 25 - 26 us for 8 - 32 tokens on the tcgen05 kernel.
 constexpr int64_t kSmallBatchMax = 8;
-static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout) {
-    (void)K;
-    return layout == POT_LAYOUT_TILED && M <= kSmallBatchMax && N % 16 == 0;
+// ... and, above four tokens, only while the eight-token activation block fits in shared memory beside the rings
+// (K <= 8192 or so): read through L2 for every unit instead, the streaming kernel loses to the tcgen05 kernel at 8
+// tokens (27.7 against 26.1 us at 13824 -> 5120) and still wins at 4 (20.3 against 25.8 us).  One token always takes
+// the GEMV kernel.
+static bool use_small(int64_t M, int64_t N, int64_t K, pot_layout_t layout, int bits = 3, int group = 128) {
+    if (layout != POT_LAYOUT_TILED || M > kSmallBatchMax || N % 16 != 0) return false;
+    if (M == 1) return true;
+    const StreamPlan p = plan_stream(N, K, M, bits, group, SK_POT, 8, 16);
+    return p.ok && (p.x_in_smem || M <= 4 || !gemm_prefill_supported(M, N, K, bits, group));
 }
 
 extern "C" size_t pot_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits, int group) {
     if (check_shape(N, K, bits, group) != POT_OK || M <= 0) return 0;
-    if (use_small(M, N, K, POT_LAYOUT_TILED)) return plan_stream(N, K, M, bits, group, SK_POT, 8, 16).ws_bytes;
+    if (use_small(M, N, K, POT_LAYOUT_TILED, bits, group)) {
+        const size_t tok8 = plan_stream(N, K, M, bits, group, SK_POT, 8, 16).ws_bytes;
+        const size_t tok1 = M == 1 ? pot_gemv_workspace_bytes(N, K, bits, group) : 0;  // one token runs the GEMV kernel
+        return tok8 > tok1 ? tok8 : tok1;
+    }
     return gemm_prefill_workspace(M, N, K, bits, group);
 }
 
@@ -151,9 +164,11 @@ static pot_status_t gemm_impl(const void* packed, const void* scales, int64_t N,
     if (!aligned16(packed) || !aligned16(scales) || !aligned16(X) || !aligned16(Y) || !aligned16(workspace))
         return POT_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;
-    if (use_small(M, N, K, layout)) {
+    if (use_small(M, N, K, layout, bits, group)) {
         const size_t need = pot_gemm_workspace_bytes(M, N, K, bits, group);
         if (need > 0 && (!workspace || ws_bytes < need)) return POT_ERR_WORKSPACE;
+        // one token: the GEMV kernel (x in every MMA column, two CTAs per SM where the share per CTA is small)
+        if (M == 1) return gemv_stream_launch(packed, scales, N, K, bits, group, X, Y, workspace, s, DT);
         const int Mi = (int)M;
 #define POT_GS(B) return launch_stream<B, SK_POT, 8, 16, 1, DT>(packed, scales, nullptr, N, K, group, X, Mi, Y, workspace, error_ptr(ERR_GEMM), s)
         if (bits == 2) POT_GS(2);

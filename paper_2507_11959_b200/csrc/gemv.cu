@@ -115,6 +115,13 @@ static pot_status_t launch_gemv_stream(const void* packed, const void* scales, c
 #undef POT_SG
 }
 
+// the tiled FP16 / BF16 GEMV for pot_gemm's single-token case
+pot_status_t gemv_stream_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group, const void* x,
+                                void* y, void* workspace, cudaStream_t s, int dt) {
+    if (dt == 0) return launch_gemv_stream<SK_POT, 0>(packed, scales, nullptr, N, K, bits, group, x, y, workspace, s);
+    return launch_gemv_stream<SK_POT, 1>(packed, scales, nullptr, N, K, bits, group, x, y, workspace, s);
+}
+
 static size_t gemv_stream_workspace(int64_t N, int64_t K, int bits, int group, int tok) {
     size_t need = 0;
     for (int occ : {1, 2}) {  // the partial-sum layout does not depend on the occupancy, the check is for safety

@@ -295,19 +295,20 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         } else {
             // chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * 8 + token: a warp reads 512
             // contiguous bytes.  Tokens >= M stay unwritten: their columns of the product are never delivered.
-            const int total = sa.M * kc;  // X is [M][K]: chunk e belongs to token e / kc
-            for (int e0 = threadIdx.x; e0 < total; e0 += 4 * W * 32) {
-                uint4 v[4];
+            // Eight consecutive threads take the same chunk of the eight tokens, so a quarter-warp stores 128 contiguous
+            // bytes (no bank conflict); each of them reads 64 contiguous bytes of its token's row with three neighbours.
+            const int total = 8 * kc;
+            for (int e0 = threadIdx.x; e0 < total; e0 += 8 * W * 32) {  // eight loads in flight per thread
+                uint4 v[8];
 #pragma unroll
-                for (int p = 0; p < 4; ++p)
-                    if (e0 + p * W * 32 < total) v[p] = ld_dependent16(src + e0 + p * W * 32);
+                for (int p = 0; p < 8; ++p) {
+                    const int e = e0 + p * W * 32, token = e & 7;
+                    if (e < total && token < sa.M) v[p] = ld_dependent16(src + (int64_t)token * kc + (e >> 3));
+                }
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    const int e = e0 + p * W * 32;
-                    if (e < total) {
-                        const int token = e / kc, i = e - token * kc;
-                        dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << 3) + token] = v[p];
-                    }
+                for (int p = 0; p < 8; ++p) {
+                    const int e = e0 + p * W * 32, token = e & 7, i = e >> 3;
+                    if (e < total && token < sa.M) dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << 3) + token] = v[p];
                 }
             }
         }
