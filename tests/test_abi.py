@@ -45,11 +45,14 @@ def test_size_helpers(L):
     assert L.pot_gemv_workspace_bytes(12288, 128, 3, 128) == 0
     ws = L.pot_gemv_workspace_bytes(4096, 11008, 3, 128)
     assert ws >= 1024 + 256 * 2 * 16 * 4 and ws % 16 == 0
-    wg = L.pot_gemm_workspace_bytes(6, 4096, 11008, 3, 128)   # small batch: eight token columns per slot
+    wg = L.pot_gemm_workspace_bytes(4, 4096, 11008, 3, 128)   # small batch: eight token columns per slot
     assert wg >= 1024 + 256 * 2 * 16 * 8 * 4 and wg % 16 == 0
-    # up to 8 tokens run the streaming kernel: one workspace size for all of them
-    assert L.pot_gemm_workspace_bytes(8, 12288, 4096, 3, 128) == L.pot_gemm_workspace_bytes(6, 12288, 4096, 3, 128)
-    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == wg
+    # 2 to 8 tokens run the streaming kernel (one workspace size for all of them) while their activations fit in
+    # shared memory; 5 to 8 tokens of a longer K run the tcgen05 kernel; one token runs the GEMV kernel
+    assert L.pot_gemm_workspace_bytes(8, 12288, 4096, 3, 128) == L.pot_gemm_workspace_bytes(2, 12288, 4096, 3, 128)
+    assert L.pot_gemm_workspace_bytes(2, 4096, 11008, 3, 128) == wg
+    assert L.pot_gemm_workspace_bytes(8, 4096, 11008, 3, 128) == 256 + 32 * 4 * 8 * 128 * 4   # (see the tcgen05 sizes below)
+    assert L.pot_gemm_workspace_bytes(1, 4096, 11008, 3, 128) >= ws
     # Larger M runs the tcgen05 kernel.  It needs scratch only for the tiles it splits along K: all of them when they
     # cover at most half of the SMs (32 tiles -> 4 splits of 32 token rows x 128 features), or those of a last
     # wave that fills at most half of the 148 CTA slots (640 tiles -> 48 tail tiles x 3 splits x 256 rows).
