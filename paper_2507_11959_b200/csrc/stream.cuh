@@ -55,6 +55,7 @@ struct StreamPlan {
     int ring_capacity;    // slots per warp that would fit
     int tok;              // B columns in use: 1 (GEMV) or 8 (small batch)
     bool x_in_smem;
+    int token_shift;      // log2 of the token slots of the staged activations (0 for the GEMV)
     size_t x_bytes, smem_bytes;
     int max_slots;        // partial-sum slots per row block
     size_t ws_counters, ws_bytes;
@@ -87,7 +88,9 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     // shared memory: header, the staged activations, W rings
     const size_t budget = (occ == 2 ? 113 : 224) * 1024;  // two CTAs per SM: 228 KB less 1 KB reserve each
     const size_t hdr = (size_t)sk_header_bytes(warps, tok);
-    const size_t xb = (size_t)(tok > 1 ? 8 : 1) * (size_t)K * 2;
+    // multi-token kernel: the staged block has 2, 4 or 8 token slots per 16-byte chunk position (the smallest that holds M)
+    p.token_shift = tok > 1 ? (M <= 2 ? 1 : (M <= 4 ? 2 : 3)) : 0;
+    const size_t xb = ((size_t)K * 2) << p.token_shift;
     // slots of 4 units unless the ring could then hold only one of them next to the staged activations
     int q = SK_QMAX;
     if (hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget) q = 2;
@@ -126,6 +129,7 @@ struct StreamArgs {
     int64_t N, K;
     uint32_t units, gw_total;      // U, grid * W
     int ncb, group, stages, x_bytes, max_slots, M;
+    int token_shift;               // log2 of the token slots of the staged activations
     int fits32;                    // U * gw_total < 2^32: 32-bit range arithmetic
     int aligned, nrb;              // row-block split (see the kernel), number of row blocks
 #ifdef SK_TRACE
@@ -293,22 +297,23 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
                 }
             }
         } else {
-            // chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * 8 + token: a warp reads 512
-            // contiguous bytes.  Tokens >= M stay unwritten: their columns of the product are never delivered.
-            // Eight consecutive threads take the same chunk of the eight tokens, so a quarter-warp stores 128 contiguous
-            // bytes (no bank conflict); each of them reads 64 contiguous bytes of its token's row with three neighbours.
-            const int total = 8 * kc;
+            // chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * T + token, T = 2, 4 or 8 token
+            // slots (the smallest that holds M): with T = 8 a warp reads 512 contiguous bytes; with fewer slots the
+            // MMA columns beyond T repeat the first T tokens and are never delivered, like the tokens >= M.  Consecutive
+            // threads take the same chunk of consecutive tokens, so a quarter-warp stores 128 contiguous bytes.
+            const int ts = sa.token_shift, tmask = (1 << ts) - 1;
+            const int total = kc << ts;
             for (int e0 = threadIdx.x; e0 < total; e0 += 8 * W * 32) {  // eight loads in flight per thread
                 uint4 v[8];
 #pragma unroll
                 for (int p = 0; p < 8; ++p) {
-                    const int e = e0 + p * W * 32, token = e & 7;
-                    if (e < total && token < sa.M) v[p] = ld_dependent16(src + (int64_t)token * kc + (e >> 3));
+                    const int e = e0 + p * W * 32, token = e & tmask;
+                    if (e < total && token < sa.M) v[p] = ld_dependent16(src + (int64_t)token * kc + (e >> ts));
                 }
 #pragma unroll
                 for (int p = 0; p < 8; ++p) {
-                    const int e = e0 + p * W * 32, token = e & 7, i = e >> 3;
-                    if (e < total && token < sa.M) dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << 3) + token] = v[p];
+                    const int e = e0 + p * W * 32, token = e & tmask, i = e >> ts;
+                    if (e < total && token < sa.M) dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << ts) + token] = v[p];
                 }
             }
         }
@@ -416,7 +421,7 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
     // ---- one unit: 2 x 32 codes of this lane -> 32 half2 (decode: needs no activations) -> eight MMAs (multiply) ----
     auto unit_ok = [&](const unsigned char* code, const unsigned char* param, uint32_t cbu) {
         return in_range(code >= ringp && code + UB <= ringp + (size_t)S * slot_bytes && param + NPARAM * PB <= ringp + (size_t)S * slot_bytes &&
-                            cbu < ncb && (!XSMEM || (size_t)(cbu + 1) * 256u * (TOK == 1 ? 1 : 8) <= (size_t)sa.x_bytes),
+                            cbu < ncb && (!XSMEM || ((size_t)(cbu + 1) * 256u << sa.token_shift) <= (size_t)sa.x_bytes),
                         err, 0x150);
     };
     auto decode = [&](const unsigned char* code, const unsigned char* param, uint32_t (&lo)[16], uint32_t (&hi)[16]) {
@@ -472,10 +477,10 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         uint32_t xq[16];
         if constexpr (XSMEM) {
             const unsigned char* xa = TOK == 1 ? xs + cbu * 256u + (uint32_t)tig * 16u
-                                               : xs + ((cbu * 16u + (uint32_t)tig) * 8u + (uint32_t)gid) * 16u;
+                                               : xs + ((((cbu * 16u + (uint32_t)tig) << sa.token_shift) + ((uint32_t)gid & ((1u << sa.token_shift) - 1u))) << 4);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 v = sk_lds128(xa + (TOK == 1 ? 64u : 512u) * i);
+                const uint4 v = sk_lds128(xa + (TOK == 1 ? 64u : (64u << sa.token_shift)) * i);
                 xq[4 * i + 0] = v.x; xq[4 * i + 1] = v.y; xq[4 * i + 2] = v.z; xq[4 * i + 3] = v.w;
             }
         } else {
@@ -591,6 +596,7 @@ inline StreamArgs stream_args(const StreamPlan& p, const void* packed, const voi
     sa.x_bytes = (int)p.x_bytes;
     sa.max_slots = p.max_slots;
     sa.M = M;
+    sa.token_shift = p.token_shift;
 #ifdef SK_TRACE
     sa.trace = g_sk_trace;
     if (g_sk_trace) g_sk_trace += 148 * 2 * 8;
