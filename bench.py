@@ -245,6 +245,7 @@ def main():
 
     if args.shard == "rows":
         sharded_rows_arm(args, B, pdist, torch, dev, stream, f16, peaks, rank, world)
+        pdist.shutdown()
         return
 
     layers3, bytes3 = build_chain(HEADLINE_BITS)
@@ -323,7 +324,7 @@ def main():
                      "per_launch_us": ms * 1e3 / max(1, launches_per_step),
                      "algorithmic_bytes_per_launch": bytes3 / max(1, launches_per_step),
                      # dram__bytes_read+write per launch from the ncu capture of the 12288x4096 launch
-                     # (profiles/ring_kernel_gemv_12288x4096_3bit.md: 1.0015 x algorithmic), scaled by bytes
+                     # (profiles/stream_kernel_gemv_12288x4096_3bit.md: 1.0015 x algorithmic), scaled by bytes
                      "traffic": NCU_TRAFFIC_RATIO * bytes3 / max(1, launches_per_step)},
     }
 
@@ -332,7 +333,8 @@ def main():
         out["cpu_baseline"] = cpu_baseline()
     del layers3
     if rank == 0:
-        print(json.dumps(out))
+        print(json.dumps(out), flush=True)
+    pdist.shutdown()
 
 
 def sharded_rows_arm(args, B, pdist, torch, dev, stream, f16, peaks, rank, world):

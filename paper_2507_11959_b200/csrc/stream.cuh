@@ -94,6 +94,12 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     // slots of 4 units unless the ring could then hold only one of them next to the staged activations
     int q = SK_QMAX;
     if (hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget) q = 2;
+    // multi-token kernel with a large activation block: three slots of 3 units rather than two of 4 (with two slots a
+    // warp has one request in flight while it works, which does not cover the latency: 18.2 against 14.0 us measured
+    // across that boundary)
+    else if (tok > 1 && hdr + xb + (size_t)warps * 3 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget &&
+             hdr + xb + (size_t)warps * 3 * (size_t)sk_slot_bytes(bits, group, kind, 3) <= budget)
+        q = 3;
     // long ranges (large matrices, one CTA per SM): slots of 8 units halve the per-slot hand-off work, if two of them fit
     else if (occ == 1 && tok == 1 && per_warp >= 32 && hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, 8) <= budget) q = 8;
     p.q = q;
@@ -297,23 +303,30 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
                 }
             }
         } else {
-            // chunk (token, unit, quarter t, part j) goes to ((unit * 4 + j) * 4 + t) * T + token, T = 2, 4 or 8 token
-            // slots (the smallest that holds M): with T = 8 a warp reads 512 contiguous bytes; with fewer slots the
-            // MMA columns beyond T repeat the first T tokens and are never delivered, like the tokens >= M.  Consecutive
-            // threads take the same chunk of consecutive tokens, so a quarter-warp stores 128 contiguous bytes.
-            const int ts = sa.token_shift, tmask = (1 << ts) - 1;
+            // T = 2, 4 or 8 token slots (the smallest that holds M).  Chunk (token, unit, quarter t, part j) goes to
+            // 16-byte slot (unit * 4 + j) * 4 T + (token / 2) * 8 + (token % 2) * 4 + t: the eight lanes of a quarter-warp
+            // of the MMA loop (tokens 2q and 2q + 1, quarters 0..3) read one 128-byte line, a warp 4 lines -- no bank
+            // conflict (token-major slots cost four-way conflicts: 11 against 8 us in the loop at 5+ tokens).  With fewer
+            // than 8 slots the MMA columns beyond T repeat the first T tokens; they are never delivered, like the
+            // tokens >= M.  The threads are numbered so that a quarter-warp also STORES one line: t fastest, then the
+            // token's parity, then j -- a warp loads the 256 contiguous bytes of a unit for two tokens.
+            const int ts = sa.token_shift;
             const int total = kc << ts;
             for (int e0 = threadIdx.x; e0 < total; e0 += 8 * W * 32) {  // eight loads in flight per thread
                 uint4 v[8];
 #pragma unroll
                 for (int p = 0; p < 8; ++p) {
-                    const int e = e0 + p * W * 32, token = e & tmask;
-                    if (e < total && token < sa.M) v[p] = ld_dependent16(src + (int64_t)token * kc + (e >> ts));
+                    const int e = e0 + p * W * 32;
+                    const int t = e & 3, par = (e >> 2) & 1, j = (e >> 3) & 3, hi = (e >> 5) & ((1 << (ts - 1)) - 1), unit_ = e >> (4 + ts);
+                    const int token = (hi << 1) | par;
+                    if (e < total && token < sa.M) v[p] = ld_dependent16(src + (int64_t)token * kc + unit_ * 16 + t * 4 + j);
                 }
 #pragma unroll
                 for (int p = 0; p < 8; ++p) {
-                    const int e = e0 + p * W * 32, token = e & tmask, i = e >> ts;
-                    if (e < total && token < sa.M) dst[((((i >> 4) * 4 + (i & 3)) * 4 + ((i >> 2) & 3)) << ts) + token] = v[p];
+                    const int e = e0 + p * W * 32;
+                    const int t = e & 3, par = (e >> 2) & 1, j = (e >> 3) & 3, hi = (e >> 5) & ((1 << (ts - 1)) - 1), unit_ = e >> (4 + ts);
+                    const int token = (hi << 1) | par;
+                    if (e < total && token < sa.M) dst[(((unit_ << 2) + j) << (2 + ts)) + (hi << 3) + (par << 2) + t] = v[p];
                 }
             }
         }
@@ -477,7 +490,8 @@ __device__ __forceinline__ void stream_body(const StreamArgs& sa, int* __restric
         uint32_t xq[16];
         if constexpr (XSMEM) {
             const unsigned char* xa = TOK == 1 ? xs + cbu * 256u + (uint32_t)tig * 16u
-                                               : xs + ((((cbu * 16u + (uint32_t)tig) << sa.token_shift) + ((uint32_t)gid & ((1u << sa.token_shift) - 1u))) << 4);
+                                               : xs + ((((cbu * 16u) << sa.token_shift) + ((((uint32_t)gid & ((1u << sa.token_shift) - 1u)) >> 1) << 3) +
+                                                        (((uint32_t)gid & 1u) << 2) + (uint32_t)tig) << 4);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 v = sk_lds128(xa + (TOK == 1 ? 64u : (64u << sa.token_shift)) * i);
@@ -619,6 +633,9 @@ pot_status_t launch_stream(const void* packed, const void* scales, const void* z
     if (p.q == 2) {
         if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2, DT>);
         return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2, DT>);
+    }
+    if constexpr (TOK > 1) {
+        if (p.q == 3) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 3, DT>);  // only chosen with x in shared memory
     }
     if constexpr (OCC == 1 && TOK == 1) {
         if (p.q == 8) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 8, DT>);  // only chosen with x in shared memory

@@ -22,6 +22,14 @@ def init(backend: str) -> tuple[int, int, int]:
     return rank, local_rank, world
 
 
+def shutdown() -> None:
+    """Leave together: a barrier, then the process group is destroyed (a rank that simply exits while another is
+    still inside a collective, or still connected to its store, makes that other rank fail at teardown)."""
+    if dist.is_initialized():
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def shard_rows(N: int, rank: int, world: int, multiple: int = 16) -> tuple[int, int]:
     """[begin, end) of the rows owned by `rank`: contiguous, multiples of `multiple`, sizes differ by
     at most one block, union = [0, N).  N must be a multiple of `multiple`."""

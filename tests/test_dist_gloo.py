@@ -36,7 +36,8 @@ def test_two_gloo_ranks_reduce_timing_and_shard():
         t = pdist.max_over_ranks(1.0 + rank)
         s = pdist.sum_over_ranks(10.0 * (rank + 1))
         lo, hi = pdist.shard_rows(4096, rank, world)
-        print(f"RESULT {rank} {t} {s} {lo} {hi}")
+        print(f"RESULT {rank} {t} {s} {lo} {hi}", flush=True)
+        pdist.shutdown()
     """ % str(ROOT))
     procs = []
     for rank in range(2):
@@ -92,7 +93,8 @@ def test_two_gloo_ranks_row_sharded_gemv_chain_equals_single_rank(oracle):
         xs = torch.cat([g1, as_t(x0[:80])])
         g2 = pdist.sharded_gemv(sh[1], xs, torch.zeros(256, dtype=torch.int32), gemv=lg)
         ok = bool(np.array_equal(as_u16(g1), y1) and np.array_equal(as_u16(g2), y2))
-        print(f"RESULT {rank} {ok} {sh[0].begin} {sh[0].end} {sh[0].even} {sh[1].even}")
+        print(f"RESULT {rank} {ok} {sh[0].begin} {sh[0].end} {sh[0].even} {sh[1].even}", flush=True)
+        pdist.shutdown()
     """ % str(ROOT))
     procs = []
     for rank in range(2):
