@@ -94,12 +94,6 @@ inline StreamPlan plan_stream(int64_t N, int64_t K, int64_t M, int bits, int gro
     // slots of 4 units unless the ring could then hold only one of them next to the staged activations
     int q = SK_QMAX;
     if (hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget) q = 2;
-    // multi-token kernel with a large activation block: three slots of 3 units rather than two of 4 (with two slots a
-    // warp has one request in flight while it works, which does not cover the latency: 18.2 against 14.0 us measured
-    // across that boundary)
-    else if (tok > 1 && hdr + xb + (size_t)warps * 3 * (size_t)sk_slot_bytes(bits, group, kind, q) > budget &&
-             hdr + xb + (size_t)warps * 3 * (size_t)sk_slot_bytes(bits, group, kind, 3) <= budget)
-        q = 3;
     // long ranges (large matrices, one CTA per SM): slots of 8 units halve the per-slot hand-off work, if two of them fit
     else if (occ == 1 && tok == 1 && per_warp >= 32 && hdr + xb + (size_t)warps * 2 * (size_t)sk_slot_bytes(bits, group, kind, 8) <= budget) q = 8;
     p.q = q;
@@ -633,9 +627,6 @@ pot_status_t launch_stream(const void* packed, const void* scales, const void* z
     if (p.q == 2) {
         if (p.x_in_smem) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 2, DT>);
         return run(stream_kernel<BITS, KIND, TOK, false, W, OCC, 2, DT>);
-    }
-    if constexpr (TOK > 1) {
-        if (p.q == 3) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 3, DT>);  // only chosen with x in shared memory
     }
     if constexpr (OCC == 1 && TOK == 1) {
         if (p.q == 8) return run(stream_kernel<BITS, KIND, TOK, true, W, OCC, 8, DT>);  // only chosen with x in shared memory
