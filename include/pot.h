@@ -186,6 +186,14 @@ pot_status_t pot_dequant(const void* packed, const void* scales_f16, int64_t N, 
  * run to run).  Canonical layout: a CUDA-core kernel with warp-shuffle reduction.
  *   x_f16 [K], y_f16 [N]; workspace >= pot_gemv_workspace_bytes(N,K,bits,group), 16-byte aligned
  *   (may be NULL when that size is 0).  `layout` says how `packed` is arranged.
+ * Ordering on the stream: the fused kernels (pot_gemv, pot_gemm, uint_gemv and their BF16 forms) are launched so that
+ * they may START while the previous kernel of the stream is still draining; they fetch codes and scales at once and
+ * wait for that kernel to end before they read x or write y and the workspace.  x, y and the workspace may therefore
+ * be produced / still be in use by the preceding call; the CODES AND SCALES MUST BE COMPLETE before the preceding
+ * kernel of the stream starts.  Every kernel of this library that writes codes or scales (pot_quantize_ref,
+ * pot_repack, pot_repack_scales, the uint_ forms) keeps its successors from starting early, so call sequences built
+ * from this library are always safe; a caller who writes codes or scales with a kernel of their own that releases its
+ * dependents early (programmatic dependent launch) must synchronise before the first GEMV that reads them.
  */
 pot_status_t pot_gemv(const void* packed, const void* scales_f16, int64_t N, int64_t K, int bits,
                       int group, pot_layout_t layout, const void* x_f16, void* y_f16,
@@ -240,8 +248,9 @@ pot_status_t pot_gemv_noalloc(const void* packed_tiled, const void* scales_f16, 
 /*
  * pot_gemm -- the matrix product that the dequantized weights feed (Sec. 4.2, last paragraph; reconstruction by
  * Eq. 1, decode by the integer add of Sec. 4.2): Y = X W~^T for M tokens: X_f16 [M,K] row-major, Y_f16 [M,N] row-major, FP32
- * accumulation, FP16 output.  M <= 8 (decode batches) runs the streaming tensor-core kernel of
- * pot_gemv with one token per MMA column, the weights decoded straight into MMA fragments;
+ * accumulation, FP16 output.  M = 1 runs pot_gemv's kernel.  2 <= M <= 8 (decode batches) runs the streaming
+ * tensor-core kernel of pot_gemv with one token per MMA column, the weights decoded straight into MMA
+ * fragments (5 <= M <= 8 only while 16 K bytes of activations fit in shared memory beside the rings: K <= 8192 or so);
  * larger M runs the tcgen05 kernel: TMA loads of X tiles, weights decoded into swizzled shared-memory tiles,
  * accumulators in tensor memory (two issuing threads with an accumulator each, added in a fixed
  * order: the result does not depend on timing); the tiles of a last, at most half-filled wave

@@ -11,7 +11,9 @@
 // of an 8-bit float with five exponent bits: exponent bits from bit 2 upwards, sign at bit 7
 // (five above the exponent's low bit), after a rotation of the word:
 //   * as FP8 operand : (rot(w) & mask) | 0x40..  is the byte pattern of +-2^(E+1) -- one
-//                      logic operation per four weights (no kernel in this tree consumes that form yet);
+//                      logic operation per four weights.  No kernel in this tree consumes that form: FP8 GEMVs built on
+//                      it (warp-level m16n8k32 MMAs, which this GPU emulates with conversions on the ALUs, and
+//                      tcgen05 MMAs with the weights in tensor memory) were exact but slower than the FP16 route;
 //   * as FP16 pair   : (rot(w) & mask16) * 2^8 + scale  (lanes 0, 2)  and
 //                      (rot(w) & mask16 << 8) + scale   (lanes 1, 3)  -- the mask / shift /
 //                      integer add into the scale's bit pattern of Sec. 4.2 of the paper.

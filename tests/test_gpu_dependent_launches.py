@@ -97,3 +97,35 @@ def test_eager_chain_without_synchronisation_follows_its_input(oracle):
         torch.cuda.synchronize()
         assert torch.equal(out, ref[r]), (it, r)
     assert B.pot_debug_errors() == (0, 0, 0)
+
+
+def test_weights_written_just_before_the_gemv_are_complete(oracle):
+    """The fused kernels fetch codes and scales before they wait for their predecessor, so the kernels that WRITE codes
+    and scales must not let their successors start early: quantize -> repack -> repack_scales -> GEMV on one stream,
+    nothing synchronised in between, new weights every time, against the same sequence run step by step."""
+    bits, G, N, K, R = 3, 128, 4096, 4096, 6
+    x = f16_dev(synth.activations(synth.rng_for(8, 300), 1, K)[0])
+    ws = B.new_workspace(B.pot_gemv_workspace_bytes(N, K, bits, G), DEV)
+    Ws = [f16_dev(synth.weights(synth.rng_for(8, 310 + r), N, K, "t5")) for r in range(R)]
+
+    def run(W, sync):
+        packed, S = B.pot_quantize_ref(W, bits, G, B.SCALE_TOP)
+        if sync:
+            torch.cuda.synchronize()
+        tiled = B.pot_repack(packed, K, bits, 0)
+        tS = B.pot_repack_scales(S, K, G, 0)
+        if sync:
+            torch.cuda.synchronize()
+        y = B.pot_gemv(tiled, tS, K, bits, G, x, B.TILED, workspace=ws)
+        torch.cuda.synchronize()
+        return y, packed, S
+
+    ref = [run(W, True) for W in Ws]
+    Y, A = oracle.matmul(ref[0][1].cpu().numpy(), bits_of(ref[0][2]), K, bits, G, bits_of(x).reshape(1, K))
+    ok, worst, tight = gate(bits_of(ref[0][0]), Y[0], A[0])
+    assert ok and tight < 4.0, (worst, tight)
+    for it in range(4 * R):
+        r = (5 * it) % R
+        y, _, _ = run(Ws[r], False)
+        assert torch.equal(y, ref[r][0]), (it, r)
+    assert B.pot_debug_errors() == (0, 0, 0)
