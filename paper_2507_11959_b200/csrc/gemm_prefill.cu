@@ -20,12 +20,18 @@
 // tcgen05.ld (each warp its own 32-lane quarter), add the two issuers' sums in a fixed order, convert to FP16 and
 // store (a warp writes 32 consecutive features of one token at a time).  The weights are re-decoded once per 256-token
 // tile (M / 256 times overall), which is the price of never writing FP16 weights to HBM.
+// For K <= 16384 the decoded weight tile does not go through shared memory at all: the producers write it into tensor
+// memory (tcgen05.st, lane = weight row, 32 columns per stage behind the 256 accumulator columns) and the MMAs take
+// their A operand from there; both issuers then work on every stage, issuer J multiplying the tile by token tile J into
+// its own 128 columns (see pf_issue_at).
 // Batches of up to 64 tokens run a variant with one tile of M token rows (the TMA box holds exactly M rows, the MMA's
 // N is M rounded up to 16), eight 24 KB stages and two TMA threads.
 //
 // All mbarrier waits are bounded (see sync.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
 #include <cuda.h>
+
+#include <cstdlib>
 
 #include <type_traits>
 
@@ -48,8 +54,10 @@ constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
 // a stage: MT X tiles (token tiles) + one weight tile
 // (the one-tile kernel serves up to PF_SMALL_TOKENS tokens: 8 KB of X per stage, so that eight stages fit)
 __host__ __device__ constexpr int pf_x_bytes(int mt) { return mt == 1 ? PF_SMALL_TOKENS * 128 : mt * PF_ATOM_BYTES; }
-__host__ __device__ constexpr int pf_stage_bytes(int mt) { return pf_x_bytes(mt) + PF_ATOM_BYTES; }
-constexpr size_t pf_smem_bytes(int stages, int mt) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt) + 256 /*barriers*/; }
+// (at = 1: the decoded weight tile lives in tensor memory, a stage of shared memory holds the X tiles only)
+__host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0) { return pf_x_bytes(mt) + (at ? 0 : PF_ATOM_BYTES); }
+constexpr size_t pf_smem_bytes(int stages, int mt, int at = 0) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt, at) + 256 /*barriers*/; }
+constexpr int PF_AT_ACC_COLS = 256;   // at = 1: accumulator columns (token t of the tile = column t), then 32 columns per stage of A
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128 (the weight rows of the tile are the
 // A operand), N = n token rows of the X tile (the B operand), 16 <= n <= 256, n % 16 == 0
@@ -119,6 +127,67 @@ __device__ __forceinline__ void pf_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "memory");
 }
 
+// tcgen05.mma with the A operand in tensor memory (lane = row of A, one 32-bit column = two K elements)
+__device__ __forceinline__ void pf_mma_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(blo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void pf_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,"
+        "%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+}
+
+// Issuer J of the variant that keeps the decoded weight tile in tensor memory: it takes EVERY stage, multiplies the tile
+// (A, from tensor memory: 128 weight rows x 64) by token tile J of the stage (B, 128 tokens, from shared memory) and
+// accumulates into columns 128 J .. 128 J + 127 -- the two issuers share the weight tile and never the accumulator, so
+// the order of the additions is fixed.  A stage is free again when every active issuer's MMAs on it have completed.
+template <int J, int PF_STAGES, int DT>
+__device__ __forceinline__ void pf_issue_at(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, int* err) {
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
+    const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
+    uint32_t blo[PF_STAGES];
+#pragma unroll
+    for (int s = 0; s < PF_STAGES; ++s)
+        blo[s] = (uint32_t)pf_smem_desc(smem0 + (uint32_t)s * pf_stage_bytes(PF_MT, 1) + (uint32_t)J * PF_ATOM_BYTES);
+    constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
+    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BM);
+    const uint32_t a0 = tmem_base + (uint32_t)PF_AT_ACC_COLS;
+    const uint32_t idesc = pf_idesc(PF_BM, DT);
+    uint32_t ready = mbar_test(full(0), 0);
+    uint32_t ph = 0;
+    for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
+#pragma unroll
+        for (int s = 0; s < PF_STAGES; ++s) {
+            const int kb = kb0 + s;
+            if (kb >= nkb) break;
+            if (!ready && !mbar_wait(full(s), ph)) {
+                if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+            }
+            ready = 0;
+            if (kb + 1 < nkb) ready = mbar_test(full((s + 1) % PF_STAGES), s + 1 >= PF_STAGES ? ph ^ 1u : ph);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int ks = 0; ks < PF_BK / 16; ++ks)
+                pf_mma_ta(d0, a0 + (uint32_t)(32 * s + 8 * ks), blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, idesc,
+                          (s != 0 || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
+            pf_commit(empty(s));
+        }
+    }
+    pf_commit(accum);
+}
+
 // The MMA issuer J of NI (one thread): takes the stages kb = J, J + NI, ... of the CTA's nkb stages and accumulates them
 // into its own accumulator (128 weight rows = lanes, n_tok token columns).  One thread's dependent instructions retire every ~5 cycles and the tensor pipe
 // idles meanwhile, so what the loop needs per MMA is prepared first: the low descriptor word of every stage's tiles (the
@@ -170,7 +239,10 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
 // Instantiated as <bits, 4, 4, 2, 2> (M > 64: 256-token tiles, four 48 KB stages) and <bits, 8, 4, 2, 1> (M <= 64: one
 // tile of up to 64 tokens, eight 24 KB stages -- a stage buffer's round trip producer -> issuer -> tensor pipe ->
 // producer is ~2000 cycles whatever the tile holds, so more buffers = more stages per unit of time).
-template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0>  // DT = 1: BF16 activations, weights and output
+// AT = 1 (MT = 2, NI = 2 only): the producers write the decoded weight tile into tensor memory (tcgen05.st) instead of
+// shared memory and the MMAs take their A operand from there, which removes a third of the shared-memory traffic of a
+// stage (16 KB written + 16 KB read of 96 KB); see pf_issue_at for the issuers' division of work.
+template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0, int AT = 0>  // DT = 1: BF16 activations, weights and output
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
@@ -179,7 +251,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int STAGE_BYTES = pf_stage_bytes(MT);
+    static_assert(AT == 0 || (MT == 2 && NI == 2), "the tensor-memory weight tile is built for 256-token tiles and two issuers");
+    constexpr int STAGE_BYTES = pf_stage_bytes(MT, AT);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PF_STAGES + 1);
@@ -190,7 +263,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
 
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
-    constexpr int TMEM_COLS = NI * PF_BN * MT;          // MT accumulators per issuer
+    constexpr int TMEM_COLS = AT ? 512 : NI * PF_BN * MT;  // MT accumulators per issuer; AT: 256 accumulator columns + the A ring
     static_assert(NG % 2 == 0 && PF_STAGES % NI == 0 && PF_STAGES % NG == 0,
                   "a group always decodes the same half of a column block; a stage buffer belongs to one issuer and one group");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -226,9 +299,9 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
             mbar_init(full(s), 1 + 4);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
-            mbar_init(empty(s), 1);
+            mbar_init(empty(s), AT ? n_mt : 1);  // AT: every active issuer reads every stage
         }
-        mbar_init(accum, NI);
+        mbar_init(accum, AT ? n_mt : NI);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // allocate the accumulator columns of tensor memory (whole warp), base address lands in shared memory
@@ -269,8 +342,13 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
-            else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            if constexpr (AT) {
+                if (warp == 1) pf_issue_at<0, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
+                else if (n_mt == 2) pf_issue_at<1, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
+            } else {
+                if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+                else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+            }
         }
     } else if (warp >= PROD_WARP0) {
         // ---------------- dequant producers (then epilogue) ---------------------------------------------
@@ -324,10 +402,34 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
                     __syncwarp();
                 }
-                unsigned char* brow = smem + (size_t)s * STAGE_BYTES + pf_x_bytes(MT) + row * 128;
                 uint32_t s16 = sc2[buf];
                 if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
                 const uint32_t s2 = s16 * 0x10001u;  // scale pattern in both halves
+                if constexpr (AT) {
+                    // the row's 64 weights of this stage = 32 packed pairs = 32 columns of this thread's tensor-memory lane
+                    uint32_t wa[32];
+#pragma unroll
+                    for (int T2 = 0; T2 < 2; ++T2) {
+                        uint32_t w2[16];
+                        if (row_ok) {
+                            if (DT == 0) potl::pot_decode32<BITS, 2>(rec[buf], T2, s2, w2);
+                            else potl::pot_decode32_bf16<BITS, 2>(rec[buf], T2, s2, w2);
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) w2[q] = 0u;
+                        }
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) wa[16 * T2 + q] = w2[q];
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");  // (behind the wait for the stage)
+                    pf_st32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(PF_AT_ACC_COLS + 32 * s), wa);
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full(s));
+                    continue;
+                }
+                unsigned char* brow = smem + (size_t)s * STAGE_BYTES + pf_x_bytes(MT) + row * 128;
 #pragma unroll
                 for (int T2 = 0; T2 < 2; ++T2) {
                     uint32_t w2[16];
@@ -374,7 +476,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
-            if (NI == 2) {                        // add the second issuer's sums (odd K blocks) to the first's: a fixed order
+            if (NI == 2 && !AT) {                 // add the second issuer's sums (odd K blocks) to the first's: a fixed order
                 uint32_t v1[32];
                 pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BM * MT + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -508,6 +610,19 @@ size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) { retur
 
 static int* prefill_error_ptr();
 
+// Where the large-M kernel keeps the decoded weight tile.  Tensor memory (the producers write it with tcgen05.st, the
+// MMAs read their A operand there) takes a third of the traffic off shared memory and measured 2 - 3 % faster on
+// K = 8192 (70B qkv and gate / up) and 1 % slower on K = 28672 (70B down), where the per-tile costs it shortens weigh
+// less than the issuers' second barrier round per stage.  FP16 only (the BF16 route keeps the shared-memory tile).
+// POT_PREFILL_WEIGHT_TILE = smem | tmem overrides the choice (a diagnostic switch: the tests run both).
+static bool prefill_weight_tile_in_tmem(int64_t K) {
+    if (const char* e = getenv("POT_PREFILL_WEIGHT_TILE")) {
+        if (e[0] == 't') return true;
+        if (e[0] == 's') return false;
+    }
+    return K <= 16384;
+}
+
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
                                  const void* X, int64_t M, void* Y, void* workspace, size_t ws_bytes, cudaStream_t s, int dt) {
     const PrefillPlan pl = prefill_plan(M, N, K);
@@ -526,8 +641,8 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
     const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits));
-    auto run = [&](auto kernel, int stages, int mt) -> pot_status_t {
-        const size_t smem = pf_smem_bytes(stages, mt);
+    auto run = [&](auto kernel, int stages, int mt, int at = 0) -> pot_status_t {
+        const size_t smem = pf_smem_bytes(stages, mt, at);
         const dim3 block((unsigned)pf_threads(4, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
@@ -548,6 +663,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1>, 8, 1);
         return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1>, 8, 1);
+    }
+    if (prefill_weight_tile_in_tmem(K)) {
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
+        return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
     }
     if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2>, 4, 2);
     if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2>, 4, 2);

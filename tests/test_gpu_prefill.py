@@ -22,9 +22,17 @@ SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20
           (64, 272, 1152), (9, 48, 2048), (65, 160, 1152)]
 
 
+@pytest.fixture(params=["smem", "tmem"])
+def weight_tile(request, monkeypatch):
+    """The large-M kernel keeps the decoded weight tile in shared memory or in tensor memory (chosen by K in production):
+    the parity tests run both through the library's diagnostic switch."""
+    monkeypatch.setenv("POT_PREFILL_WEIGHT_TILE", request.param)
+    return request.param
+
+
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("G", [64, 128])
-def test_prefill_gemm_matches_oracle(B, oracle, bits, G):
+def test_prefill_gemm_matches_oracle(B, oracle, bits, G, weight_tile):
     for i, (M, N, K) in enumerate(SHAPES):
         c = PotCase(N, K, bits, G, dist="normal", sigma=0.015, seed=(5, 10 * bits + i))
         X = synth.activations(synth.rng_for(5, 100 + i), M, K, outliers=(i % 2 == 1))
@@ -35,7 +43,7 @@ def test_prefill_gemm_matches_oracle(B, oracle, bits, G):
         assert ok and tight < 4.0, (M, N, K, worst, tight)
 
 
-def test_split_k_workspace_is_reusable(B, oracle):
+def test_split_k_workspace_is_reusable(B, oracle, weight_tile):
     """Few tiles and a deep K: the kernel splits K (8 ways here), adds the splits in a fixed order and leaves its
     arrival counters at zero -- two calls on one workspace give the same bits, equal to the oracle within the gate."""
     bits, G, M, N, K = 3, 128, 40, 384, 4096
@@ -54,9 +62,10 @@ def test_split_k_workspace_is_reusable(B, oracle):
     assert ok and tight < 4.0, (worst, tight)
 
 
-def test_two_issuers_give_the_same_bits_every_time(B, oracle):
-    """The two MMA issuers accumulate alternate K blocks into separate accumulators that the epilogue adds in a fixed
-    order: nothing in the result may depend on which of them ran first."""
+def test_two_issuers_give_the_same_bits_every_time(B, oracle, weight_tile):
+    """The two MMA issuers accumulate into separate accumulators (alternate K blocks, added by the epilogue in a fixed
+    order; or, with the weight tile in tensor memory, one token tile each): nothing in the result may depend on which of
+    them ran first."""
     bits, G, M, N, K = 3, 128, 300, 272, 2304
     c = PotCase(N, K, bits, G, dist="t5", seed=(5, 88))
     dX = f16_dev(synth.activations(synth.rng_for(5, 188), M, K, outliers=True))
@@ -68,7 +77,7 @@ def test_two_issuers_give_the_same_bits_every_time(B, oracle):
 
 
 @pytest.mark.parametrize("bits", [3])
-def test_prefill_one_hot_tokens_return_dequantized_columns(B, oracle, bits):
+def test_prefill_one_hot_tokens_return_dequantized_columns(B, oracle, bits, weight_tile):
     """token t = e_{k_t}: row t of Y must equal column k_t of the dequantized matrix bit for bit."""
     G, N, K, M = 128, 256, 640, 160
     c = PotCase(N, K, bits, G, dist="normal", seed=(5, 60))
