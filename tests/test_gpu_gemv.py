@@ -93,8 +93,10 @@ def test_uint_gemv_matches_oracle(B, oracle, bits, G):
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
-@pytest.mark.parametrize("M", [1, 4, 8, 13, 16, 32])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 7, 8, 13, 16, 32])
 def test_pot_gemm_small_batch_matches_oracle(B, oracle, bits, M):
+    """M = 1: the GEMV kernel; 2 / 3-4 / 5-8 tokens: the streaming kernel with 2 / 4 / 8 token slots (K = 11008 at 5-8
+    tokens: the tcgen05 kernel, its activation block does not fit in shared memory); above: the tcgen05 kernel."""
     G = 128
     for i, (N, K) in enumerate([(48, 640), (256, 4096), (64, 11008)]):
         c = PotCase(N, K, bits, G, dist="t5", seed=(4, 500 + 10 * bits + i))
