@@ -20,10 +20,12 @@
 // tcgen05.ld (each warp its own 32-lane quarter), add the two issuers' sums in a fixed order, convert to FP16 and
 // store (a warp writes 32 consecutive features of one token at a time).  The weights are re-decoded once per 256-token
 // tile (M / 256 times overall), which is the price of never writing FP16 weights to HBM.
-// For K <= 16384 the decoded weight tile does not go through shared memory at all: the producers write it into tensor
-// memory (tcgen05.st, lane = weight row, 32 columns per stage behind the 256 accumulator columns) and the MMAs take
-// their A operand from there; both issuers then work on every stage, issuer J multiplying the tile by token tile J into
-// its own 128 columns (see pf_issue_at).
+// By default the decoded weight tile of the large-M kernel does not go through shared memory at all (AT = 1): the
+// producers -- two groups then -- write it into tensor memory (tcgen05.st, lane = weight row, 32 columns per stage behind
+// the 256 accumulator columns) and the MMAs take their A operand from there; a stage of shared memory holds X only (six
+// stages of 32 KB); both issuers work on every stage, issuer J multiplying the tile by token tile J into its own 128
+// columns (see pf_issue_at).  The description above is the shared-memory-tile kernel, kept for the one-token-tile
+// variant and as a selectable alternative.
 // Batches of up to 64 tokens run a variant with one tile of M token rows (the TMA box holds exactly M rows, the MMA's
 // N is M rounded up to 16), eight 24 KB stages and two TMA threads.
 //
@@ -241,8 +243,11 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
 // producer is ~2000 cycles whatever the tile holds, so more buffers = more stages per unit of time).
 // AT = 1 (MT = 2, NI = 2 only): the producers write the decoded weight tile into tensor memory (tcgen05.st) instead of
 // shared memory and the MMAs take their A operand from there, which removes a third of the shared-memory traffic of a
-// stage (16 KB written + 16 KB read of 96 KB); see pf_issue_at for the issuers' division of work.
-template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0, int AT = 0>  // DT = 1: BF16 activations, weights and output
+// stage (16 KB written + 16 KB read of 96 KB); see pf_issue_at for the issuers' division of work.  Instantiated as
+// <bits, 6, 2, 2, 2, dt, 1>: 256 accumulator columns + 6 x 32 columns of A = 448 of the 512 columns.
+// NGP of the NG groups decode, the others only take part in the epilogue (measured slower than NGP = NG = 2 -- the
+// waiting groups poll the accumulator barrier through the whole main loop -- and not instantiated).
+template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0, int AT = 0, int NGP = NG>  // DT = 1: BF16 activations, weights and output
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
@@ -264,7 +269,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
     constexpr int TMEM_COLS = AT ? 512 : NI * PF_BN * MT;  // MT accumulators per issuer; AT: 256 accumulator columns + the A ring
-    static_assert(NG % 2 == 0 && PF_STAGES % NI == 0 && PF_STAGES % NG == 0,
+    static_assert(NGP % 2 == 0 && NGP <= NG && PF_STAGES % NI == 0 && PF_STAGES % NGP == 0,
                   "a group always decodes the same half of a column block; a stage buffer belongs to one issuer and one group");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
@@ -381,17 +386,17 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
             }
         };
-        const int nmine = nkb > grp ? (nkb - grp + NG - 1) / NG : 0;   // stages kb = grp, grp + NG, ...
+        const int nmine = (grp < NGP && nkb > grp) ? (nkb - grp + NGP - 1) / NGP : 0;   // stages kb = grp, grp + NGP, ...
 #pragma unroll
         for (int p = 0; p < PF_DEPTH - 1; ++p)
-            if (p < nmine) load(NG * p + grp, p);
+            if (p < nmine) load(NGP * p + grp, p);
         for (int i4 = 0; i4 < nmine; i4 += PF_DEPTH) {
 #pragma unroll
             for (int buf = 0; buf < PF_DEPTH; ++buf) {
                 const int i = i4 + buf;
                 if (i >= nmine) break;
-                const int kb = NG * i + grp;
-                if (i + PF_DEPTH - 1 < nmine) load(kb + NG * (PF_DEPTH - 1), (buf + PF_DEPTH - 1) % PF_DEPTH);
+                const int kb = NGP * i + grp;
+                if (i + PF_DEPTH - 1 < nmine) load(kb + NGP * (PF_DEPTH - 1), (buf + PF_DEPTH - 1) % PF_DEPTH);
                 const int s = kb % PF_STAGES;
                 if (kb >= PF_STAGES) {
                     // Every lane polls (the warp is about to WRITE the stage).  One polling lane + __syncwarp() left the
@@ -462,7 +467,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         // bounds: control flow added to them costs the tensor pipe several per cent.)
         const bool gave_up = err != nullptr && *reinterpret_cast<volatile int*>(err) != 0;
         // Lane = weight row (feature), column = token.  Warp (q, part): features n0 + 32 q .. + 31 (a warp may only touch its
-        // own quarter of the lanes), token columns part * 32 MT .. + 32 MT - 1.
+        // own quarter of the lanes), token columns part * 32 CH .. + 32 CH - 1 (CH chunks of 32 per warp).
         const int q = warp & 3;
         const int part = (warp - PROD_WARP0) >> 2;
         const int64_t feat = n0 + 32 * q + lane;
@@ -470,9 +475,11 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         item(tile, zsplit, splits);
         const int tail_index = tile - n_full;   // index of the tile among the split ones
         const int64_t rows_alloc = M < PF_BM * MT ? M : PF_BM * MT;  // token rows kept per tile in the workspace
+        constexpr int CH = (MT * PF_BM / 32) / NG;   // 32-column chunks per warp: the NG warps of a lane quarter share the tile's columns
+        static_assert(CH * NG * 32 == MT * PF_BM, "the epilogue warps must cover every token column");
 #pragma unroll
-        for (int cc = 0; cc < MT; ++cc) {
-            const int col = (part * MT + cc) * 32;
+        for (int cc = 0; cc < CH; ++cc) {
+            const int col = (part * CH + cc) * 32;
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
@@ -610,17 +617,14 @@ size_t gemm_prefill_workspace(int64_t M, int64_t N, int64_t K, int, int) { retur
 
 static int* prefill_error_ptr();
 
-// Where the large-M kernel keeps the decoded weight tile.  Tensor memory (the producers write it with tcgen05.st, the
-// MMAs read their A operand there) takes a third of the traffic off shared memory and measured 2 - 3 % faster on
-// K = 8192 (70B qkv and gate / up) and 1 % slower on K = 28672 (70B down), where the per-tile costs it shortens weigh
-// less than the issuers' second barrier round per stage.  FP16 only (the BF16 route keeps the shared-memory tile).
-// POT_PREFILL_WEIGHT_TILE = smem | tmem overrides the choice (a diagnostic switch: the tests run both).
-static bool prefill_weight_tile_in_tmem(int64_t K) {
-    if (const char* e = getenv("POT_PREFILL_WEIGHT_TILE")) {
-        if (e[0] == 't') return true;
-        if (e[0] == 's') return false;
-    }
-    return K <= 16384;
+// Where the large-M kernel keeps the decoded weight tile: in tensor memory (the producers write it with tcgen05.st, the
+// MMAs read their A operand there).  That takes a third of the traffic off shared memory, and a stage of shared memory
+// then holds X only, so six stages fit instead of four, and two producer groups keep up: measured 0.85 - 0.88 of the
+// cuBLAS burst figure on the six 70B points against 0.80 - 0.86 with the tile in shared memory (four stages, four
+// groups).  POT_PREFILL_WEIGHT_TILE = smem selects the shared-memory kernel (a diagnostic switch: the tests run both).
+static bool prefill_weight_tile_in_tmem() {
+    const char* e = getenv("POT_PREFILL_WEIGHT_TILE");
+    return !(e && e[0] == 's');
 }
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -641,9 +645,9 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
     const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits));
-    auto run = [&](auto kernel, int stages, int mt, int at = 0) -> pot_status_t {
+    auto run = [&](auto kernel, int stages, int mt, int at = 0, int ng = 4) -> pot_status_t {
         const size_t smem = pf_smem_bytes(stages, mt, at);
-        const dim3 block((unsigned)pf_threads(4, 2));
+        const dim3 block((unsigned)pf_threads(ng, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (uint16_t*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
@@ -655,6 +659,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
             if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1, 1>, 8, 1);
             return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1, 1>, 8, 1);
         }
+        if (prefill_weight_tile_in_tmem()) {
+            if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 2, 2, 2, 1, 1>, 6, 2, 1, 2);
+            if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 2, 2, 2, 1, 1>, 6, 2, 1, 2);
+            return run(pot_gemm_prefill_kernel<4, 6, 2, 2, 2, 1, 1>, 6, 2, 1, 2);
+        }
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2, 1>, 4, 2);
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 1>, 4, 2);
         return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 1>, 4, 2);
@@ -664,10 +673,10 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1>, 8, 1);
         return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1>, 8, 1);
     }
-    if (prefill_weight_tile_in_tmem(K)) {
-        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
-        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
-        return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 0, 1>, 4, 2, 1);
+    if (prefill_weight_tile_in_tmem()) {  // two producer groups, six stages (32 KB of X each), the A ring in tensor memory
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 2, 2, 2, 0, 1>, 6, 2, 1, 2);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 2, 2, 2, 0, 1>, 6, 2, 1, 2);
+        return run(pot_gemm_prefill_kernel<4, 6, 2, 2, 2, 0, 1>, 6, 2, 1, 2);
     }
     if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2>, 4, 2);
     if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2>, 4, 2);
