@@ -59,7 +59,10 @@ __host__ __device__ constexpr int pf_x_bytes(int mt) { return mt == 1 ? PF_SMALL
 // (at = 1: the decoded weight tile lives in tensor memory, a stage of shared memory holds the X tiles only)
 __host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0) { return pf_x_bytes(mt) + (at ? 0 : PF_ATOM_BYTES); }
 constexpr size_t pf_smem_bytes(int stages, int mt, int at = 0) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt, at) + 256 /*barriers*/; }
-constexpr int PF_AT_ACC_COLS = 256;   // at = 1: accumulator columns (token t of the tile = column t), then 32 columns per stage of A
+constexpr int PF_AT_ACC_COLS = 256;   // at = 1, 256-token tiles: accumulator columns (token t of the tile = column t), then 32 columns per stage of A
+// at = 1, the one-tile kernel (up to 64 tokens): the two issuers' accumulators take 64 columns each, the A ring follows
+constexpr int PF_AT1_ACC_STRIDE = PF_SMALL_TOKENS;
+__host__ __device__ constexpr int pf_at_ring_col0(int mt) { return mt == 2 ? PF_AT_ACC_COLS : 2 * PF_AT1_ACC_STRIDE; }
 
 // UMMA instruction descriptor: FP16 x FP16 -> FP32, both operands K-major, M = 128 (the weight rows of the tile are the
 // A operand), N = n token rows of the X tile (the B operand), 16 <= n <= 256, n % 16 == 0
@@ -190,6 +193,43 @@ __device__ __forceinline__ void pf_issue_at(uint32_t smem0, uint32_t bar0, uint3
     pf_commit(accum);
 }
 
+// Issuer J of the one-tile kernel with the weight tile in tensor memory: as pf_issue (alternate stages, its own
+// accumulator -- 64 columns at 64 J), with the A operand taken from the stage's 32 columns of the ring.
+template <int J, int NI, int PF_STAGES, int DT>
+__device__ __forceinline__ void pf_issue_at1(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, uint32_t n_tok, int* err) {
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
+    const uint32_t accum = bar0 + 8u * (2 * PF_STAGES);
+    uint32_t blo[PF_STAGES];
+#pragma unroll
+    for (int s = 0; s < PF_STAGES; ++s) blo[s] = (uint32_t)pf_smem_desc(smem0 + (uint32_t)s * pf_stage_bytes(1, 1));
+    constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
+    const uint32_t d0 = tmem_base + (uint32_t)(J * PF_AT1_ACC_STRIDE);
+    const uint32_t a0 = tmem_base + (uint32_t)pf_at_ring_col0(1);
+    const uint32_t idesc = pf_idesc(n_tok, DT);
+    uint32_t ready = mbar_test(full(J), 0);
+    uint32_t ph = 0;
+    for (int kb0 = 0; kb0 < nkb; kb0 += PF_STAGES, ph ^= 1u) {
+#pragma unroll
+        for (int s = J; s < PF_STAGES; s += NI) {
+            const int kb = kb0 + s;
+            if (kb >= nkb) break;
+            if (!ready && !mbar_wait(full(s), ph)) {
+                if (err) atomicCAS(err, 0, 0x20 | (kb << 8));
+            }
+            ready = 0;
+            if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int ks = 0; ks < PF_BK / 16; ++ks)
+                pf_mma_ta(d0, a0 + (uint32_t)(32 * s + 8 * ks), blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, idesc,
+                          (s != J || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
+            pf_commit(empty(s));
+        }
+    }
+    pf_commit(accum);
+}
+
 // The MMA issuer J of NI (one thread): takes the stages kb = J, J + NI, ... of the CTA's nkb stages and accumulates them
 // into its own accumulator (128 weight rows = lanes, n_tok token columns).  One thread's dependent instructions retire every ~5 cycles and the tensor pipe
 // idles meanwhile, so what the loop needs per MMA is prepared first: the low descriptor word of every stage's tiles (the
@@ -256,7 +296,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle atoms and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    static_assert(AT == 0 || (MT == 2 && NI == 2), "the tensor-memory weight tile is built for 256-token tiles and two issuers");
+    static_assert(AT == 0 || NI == 2, "the tensor-memory weight tile is built for two issuers");
+    constexpr bool AT2 = AT && MT == 2;   // both issuers on every stage, one token tile each (else: alternate stages)
     constexpr int STAGE_BYTES = pf_stage_bytes(MT, AT);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
@@ -304,9 +345,9 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
             mbar_init(full(s), 1 + 4);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
-            mbar_init(empty(s), AT ? n_mt : 1);  // AT: every active issuer reads every stage
+            mbar_init(empty(s), AT2 ? n_mt : 1);  // AT2: every active issuer reads every stage
         }
-        mbar_init(accum, AT ? n_mt : NI);
+        mbar_init(accum, AT2 ? n_mt : NI);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // allocate the accumulator columns of tensor memory (whole warp), base address lands in shared memory
@@ -347,9 +388,12 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     } else if (warp <= NI) {
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
-            if constexpr (AT) {
+            if constexpr (AT2) {
                 if (warp == 1) pf_issue_at<0, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
                 else if (n_mt == 2) pf_issue_at<1, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
+            } else if constexpr (AT) {
+                if (warp == 1) pf_issue_at1<0, NI, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
+                else pf_issue_at1<NI - 1, NI, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
             } else {
                 if (NI == 1 || warp == 1) pf_issue<0, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
                 else pf_issue<NI - 1, NI, PF_STAGES, MT, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
@@ -427,7 +471,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                         for (int q = 0; q < 16; ++q) wa[16 * T2 + q] = w2[q];
                     }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");  // (behind the wait for the stage)
-                    pf_st32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(PF_AT_ACC_COLS + 32 * s), wa);
+                    pf_st32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(pf_at_ring_col0(MT) + 32 * s), wa);
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
@@ -483,9 +527,9 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
-            if (NI == 2 && !AT) {                 // add the second issuer's sums (odd K blocks) to the first's: a fixed order
+            if (NI == 2 && !AT2) {                // add the second issuer's sums (odd K blocks) to the first's: a fixed order
                 uint32_t v1[32];
-                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(PF_BM * MT + col), v1);
+                pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)((AT ? PF_AT1_ACC_STRIDE : PF_BM * MT) + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
@@ -667,6 +711,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 4, 4, 2, 2, 1>, 4, 2);
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 1>, 4, 2);
         return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 1>, 4, 2);
+    }
+    if (M <= PF_SMALL_TOKENS && prefill_weight_tile_in_tmem()) {  // twelve 8 KB stages of X, the A ring fills tensor memory
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
+        return run(pot_gemm_prefill_kernel<4, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
     }
     if (M <= PF_SMALL_TOKENS) {
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
