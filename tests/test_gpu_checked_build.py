@@ -18,7 +18,8 @@ def test_small_shape_suite_against_the_checked_build():
     lib = build.build(checked=True)
     env = dict(os.environ, POT_B200_LIB=str(lib))
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
-           "tests/test_gpu_gemv.py", "tests/test_gpu_prefill.py", "tests/test_gpu_dequant.py", "tests/test_zz_no_alloc.py"]
+           "tests/test_gpu_gemv.py", "tests/test_gpu_prefill.py", "tests/test_gpu_dequant.py", "tests/test_gpu_bf16.py",
+           "tests/test_gpu_dependent_launches.py", "tests/test_zz_no_alloc.py"]
     r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
     assert " passed" in r.stdout and "failed" not in r.stdout, r.stdout[-1000:]
