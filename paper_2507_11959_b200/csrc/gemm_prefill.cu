@@ -342,6 +342,40 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const int nkb = (int)(2 * (cb1 - cb0));
     const int kb0 = (int)(2 * cb0);
 
+    // ---- dequant producers, part 1 (before the set-up below, so that the first loads of codes and scales -- constants,
+    // they do not depend on the previous kernel -- are in flight while the barriers and the tensor memory are set up and
+    // the kernel waits for its predecessor): thread = one weight row; group g owns the stages with kb % NGP == g, hence
+    // (NGP is even) always the same half of the records.
+    const int pt = threadIdx.x - 32 * PROD_WARP0;          // 0 .. NPT-1 for the producer warps
+    const int grp = pt >> 7, row = pt & 127, half = grp & 1;
+    const int64_t n = n0 + row;
+    const bool row_ok = n < N;
+    const int64_t rb = n >> 4;
+    const int r = (int)(n & 15);
+    const int spg = 128 / G;
+    // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.  Every 16-byte plane of the
+    // row holds one word of each quarter; the group needs quarters 2*grp and 2*grp + 1: 8 bytes per plane.
+    constexpr int PF_DEPTH = 4;
+    uint32_t rec[PF_DEPTH][2 * BITS];
+    uint32_t sc2[PF_DEPTH];
+    auto load = [&](int kb, int buf) {
+        if (row_ok) {
+            const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cb0 + (kb >> 1)) * (16 * BITS));
+#pragma unroll
+            for (int t = 0; t < BITS; ++t) {
+                const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
+                rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
+            }
+            // tiled scales: the unit's values sit together, rows r and r + 8 of a group in one word
+            const int64_t so = (rb * ncb + cb0 + (kb >> 1)) * (16 * spg) + potl::scale_tile_index(r, spg == 2 ? half : 0);
+            sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
+        }
+    };
+    const int nmine = (warp >= PROD_WARP0 && grp < NGP && nkb > grp) ? (nkb - grp + NGP - 1) / NGP : 0;   // stages kb = grp, grp + NGP, ...
+#pragma unroll
+    for (int p = 0; p < PF_DEPTH - 1; ++p)
+        if (p < nmine) load(NGP * p + grp, p);
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < PF_STAGES; ++s) {
             mbar_init(full(s), 1 + 4);  // the TMA thread's expect_tx arrival + one arrival per warp of the group that fills the stage
@@ -400,40 +434,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             }
         }
     } else if (warp >= PROD_WARP0) {
-        // ---------------- dequant producers (then epilogue) ---------------------------------------------
-        // NG groups of four warps take the stages in turn: a stage visit costs a warp a fixed ~1000 cycles of
-        // hand-off latency (barrier test, proxy fence, arrive), so more stages must be in preparation at once.
-        // Stage kb covers columns 64*kb .. 64*kb+63, i.e. half (kb & 1) of column block kb / 2; group g owns the
-        // stages with kb % NG == g, hence (NG is even) always the same half of the records.  Thread = one weight row.
-        const int pt = threadIdx.x - 32 * PROD_WARP0;          // 0 .. NPT-1
-        const int grp = pt >> 7, row = pt & 127, half = grp & 1;
-        const int64_t n = n0 + row;
-        const bool row_ok = n < N;
-        const int64_t rb = n >> 4;
-        const int r = (int)(n & 15);
-        const int gpr = (int)(K / G), spg = 128 / G;
-        // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.  Every 16-byte plane of the
-        // row holds one word of each quarter; the group needs quarters 2*grp and 2*grp + 1: 8 bytes per plane.
-        constexpr int PF_DEPTH = 4;
-        uint32_t rec[PF_DEPTH][2 * BITS];
-        uint32_t sc2[PF_DEPTH];
-        auto load = [&](int kb, int buf) {
-            if (row_ok) {
-                const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cb0 + (kb >> 1)) * (16 * BITS));
-#pragma unroll
-                for (int t = 0; t < BITS; ++t) {
-                    const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
-                    rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
-                }
-                // tiled scales: the unit's values sit together, rows r and r + 8 of a group in one word
-                const int64_t so = (rb * ncb + cb0 + (kb >> 1)) * (16 * spg) + potl::scale_tile_index(r, spg == 2 ? half : 0);
-                sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
-            }
-        };
-        const int nmine = (grp < NGP && nkb > grp) ? (nkb - grp + NGP - 1) / NGP : 0;   // stages kb = grp, grp + NGP, ...
-#pragma unroll
-        for (int p = 0; p < PF_DEPTH - 1; ++p)
-            if (p < nmine) load(NGP * p + grp, p);
+        // ---------------- dequant producers, part 2 (then epilogue) -----------------------------------
+        // The groups of four warps take the stages in turn: a stage visit costs a warp a fixed ~1000 cycles of
+        // hand-off latency (barrier test, fence, arrive), so more stages must be in preparation at once.
+        // Stage kb covers columns 64*kb .. 64*kb+63, i.e. half (kb & 1) of column block kb / 2.
         for (int i4 = 0; i4 < nmine; i4 += PF_DEPTH) {
 #pragma unroll
             for (int buf = 0; buf < PF_DEPTH; ++buf) {
