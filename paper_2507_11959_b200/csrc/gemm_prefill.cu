@@ -57,7 +57,10 @@ constexpr int PF_ATOM_BYTES = 128 * 128;             // 128 rows x 64 halves
 // (the one-tile kernel serves up to PF_SMALL_TOKENS tokens: 8 KB of X per stage, so that eight stages fit)
 __host__ __device__ constexpr int pf_x_bytes(int mt) { return mt == 1 ? PF_SMALL_TOKENS * 128 : mt * PF_ATOM_BYTES; }
 // (at = 1: the decoded weight tile lives in tensor memory, a stage of shared memory holds the X tiles only)
-__host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0) { return pf_x_bytes(mt) + (at ? 0 : PF_ATOM_BYTES); }
+// K sub-blocks of 64 columns per stage: two in the one-tile kernel with the weight ring in tensor memory (a stage is then a
+// whole 128-column block: half as many stage visits per byte for every role), one otherwise
+__host__ __device__ constexpr int pf_bks(int mt, int at) { return (mt == 1 && at) ? 2 : 1; }
+__host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0) { return pf_x_bytes(mt) * pf_bks(mt, at) + (at ? 0 : PF_ATOM_BYTES); }
 constexpr size_t pf_smem_bytes(int stages, int mt, int at = 0) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt, at) + 256 /*barriers*/; }
 constexpr int PF_AT_ACC_COLS = 256;   // at = 1, 256-token tiles: accumulator columns (token t of the tile = column t), then 32 columns per stage of A
 // at = 1, the one-tile kernel (up to 64 tokens): the two issuers' accumulators take 64 columns each, the A ring follows
@@ -110,6 +113,11 @@ __device__ __forceinline__ void pf_mma2(uint32_t d_tmem, uint32_t alo, uint32_t 
 __device__ __forceinline__ uint2 pf_ldg_v2(const uint2* p) {
     uint2 v;
     asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint4 pf_ldg_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
 __device__ __forceinline__ uint32_t pf_ldg_u16(const uint16_t* p) {
@@ -204,6 +212,8 @@ __device__ __forceinline__ void pf_issue_at1(uint32_t smem0, uint32_t bar0, uint
 #pragma unroll
     for (int s = 0; s < PF_STAGES; ++s) blo[s] = (uint32_t)pf_smem_desc(smem0 + (uint32_t)s * pf_stage_bytes(1, 1));
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
+    constexpr int BKS = pf_bks(1, 1);                       // 64-column sub-blocks per stage
+    constexpr uint32_t SLOT = 32u * BKS;                    // tensor-memory columns of a stage's weights
     const uint32_t d0 = tmem_base + (uint32_t)(J * PF_AT1_ACC_STRIDE);
     const uint32_t a0 = tmem_base + (uint32_t)pf_at_ring_col0(1);
     const uint32_t idesc = pf_idesc(n_tok, DT);
@@ -221,8 +231,9 @@ __device__ __forceinline__ void pf_issue_at1(uint32_t smem0, uint32_t bar0, uint
             if (kb + NI < nkb) ready = mbar_test(full((s + NI) % PF_STAGES), s + NI >= PF_STAGES ? ph ^ 1u : ph);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int ks = 0; ks < PF_BK / 16; ++ks)
-                pf_mma_ta(d0, a0 + (uint32_t)(32 * s + 8 * ks), blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, idesc,
+            for (int ks = 0; ks < BKS * (PF_BK / 16); ++ks)   // sub-block ks / 4 of the stage: its own X tile, the next 32 columns of A
+                pf_mma_ta(d0, a0 + SLOT * (uint32_t)s + (uint32_t)(8 * ks),
+                          blo[s] + (uint32_t)(((ks >> 2) * pf_x_bytes(1) + (ks & 3) * 32) >> 4), desc_hi, idesc,
                           (s != J || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
             pf_commit(empty(s));
         }
@@ -298,6 +309,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     static_assert(AT == 0 || NI == 2, "the tensor-memory weight tile is built for two issuers");
     constexpr bool AT2 = AT && MT == 2;   // both issuers on every stage, one token tile each (else: alternate stages)
+    constexpr int BKS = pf_bks(MT, AT);   // 64-column sub-blocks per stage
     constexpr int STAGE_BYTES = pf_stage_bytes(MT, AT);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
@@ -310,7 +322,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
     constexpr int TMEM_COLS = AT ? 512 : NI * PF_BN * MT;  // MT accumulators per issuer; AT: 256 accumulator columns + the A ring
-    static_assert(NGP % 2 == 0 && NGP <= NG && PF_STAGES % NI == 0 && PF_STAGES % NGP == 0,
+    static_assert((NGP % 2 == 0 || BKS == 2) && NGP <= NG && PF_STAGES % NI == 0 && PF_STAGES % NGP == 0,
                   "a group always decodes the same half of a column block; a stage buffer belongs to one issuer and one group");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
@@ -339,8 +351,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const int n_mt = M - m0 > PF_BM ? MT : 1;
     // token rows the MMA reads from the X stage: whole tiles, or (one-tile kernel) the batch rounded up to the MMA's N step
     const uint32_t n_tok = MT == 1 ? (uint32_t)((M + 15) & ~(int64_t)15) : (uint32_t)(n_mt * PF_BM);  // MT == 1: M <= 64
-    const int nkb = (int)(2 * (cb1 - cb0));
-    const int kb0 = (int)(2 * cb0);
+    const int nkb = (int)((2 / BKS) * (cb1 - cb0));   // stages of this item
+    const int kb0 = (int)((2 / BKS) * cb0);
 
     // ---- dequant producers, part 1 (before the set-up below, so that the first loads of codes and scales -- constants,
     // they do not depend on the previous kernel -- are in flight while the barriers and the tensor memory are set up and
@@ -355,20 +367,33 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     const int spg = 128 / G;
     // The packed codes are prefetched PF_DEPTH - 1 of the group's stages ahead.  Every 16-byte plane of the
     // row holds one word of each quarter; the group needs quarters 2*grp and 2*grp + 1: 8 bytes per plane.
-    constexpr int PF_DEPTH = 4;
-    uint32_t rec[PF_DEPTH][2 * BITS];
-    uint32_t sc2[PF_DEPTH];
+    // (A double-width stage -- BKS = 2 -- takes the whole record: 16 bytes per plane, and both groups' scales.)
+    constexpr int PF_DEPTH = BKS == 2 ? 3 : 4;
+    uint32_t rec[PF_DEPTH][2 * BKS * BITS];
+    uint32_t sc2[PF_DEPTH][BKS];
     auto load = [&](int kb, int buf) {
         if (row_ok) {
-            const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cb0 + (kb >> 1)) * (16 * BITS));
-#pragma unroll
-            for (int t = 0; t < BITS; ++t) {
-                const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
-                rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
-            }
+            const int64_t cbx = cb0 + (BKS == 2 ? kb : (kb >> 1));   // the stage's column block
             // tiled scales: the unit's values sit together, rows r and r + 8 of a group in one word
-            const int64_t so = (rb * ncb + cb0 + (kb >> 1)) * (16 * spg) + potl::scale_tile_index(r, spg == 2 ? half : 0);
-            sc2[buf] = pf_ldg_u16(scales + so);  // raw bits: any arithmetic here would stall on the load
+            const int64_t so = (rb * ncb + cbx) * (16 * spg);
+            if constexpr (BKS == 2) {
+                const uint4* unit = packed + (rb * ncb + cbx) * (16 * BITS);
+#pragma unroll
+                for (int t = 0; t < BITS; ++t) {
+                    const uint4 q = pf_ldg_v4(unit + t * 16 + r);
+                    rec[buf][4 * t + 0] = q.x; rec[buf][4 * t + 1] = q.y; rec[buf][4 * t + 2] = q.z; rec[buf][4 * t + 3] = q.w;
+                }
+                sc2[buf][0] = pf_ldg_u16(scales + so + potl::scale_tile_index(r, 0));
+                sc2[buf][BKS - 1] = pf_ldg_u16(scales + so + potl::scale_tile_index(r, spg == 2 ? 1 : 0));
+            } else {
+                const uint2* unit = reinterpret_cast<const uint2*>(packed + (rb * ncb + cbx) * (16 * BITS));
+#pragma unroll
+                for (int t = 0; t < BITS; ++t) {
+                    const uint2 q = pf_ldg_v2(unit + (t * 16 + r) * 2 + half);
+                    rec[buf][2 * t + 0] = q.x; rec[buf][2 * t + 1] = q.y;
+                }
+                sc2[buf][0] = pf_ldg_u16(scales + so + potl::scale_tile_index(r, spg == 2 ? half : 0));  // raw bits: any arithmetic here would stall on the load
+            }
         }
     };
     const int nmine = (warp >= PROD_WARP0 && grp < NGP && nkb > grp) ? (nkb - grp + NGP - 1) / NGP : 0;   // stages kb = grp, grp + NGP, ...
@@ -412,11 +437,16 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 ready = (kn < nkb && kn >= PF_STAGES) ? mbar_test(empty(kn % PF_STAGES), (uint32_t)((kn / PF_STAGES - 1) & 1)) : 0u;
                 // MT == 1 (M <= 64): the box holds exactly the M token rows -- the TMA unit spends time on every row of a
                 // box, in range or not; the rows of the tile that nothing writes belong to tokens that are never stored
-                mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u : (uint32_t)n_mt * PF_ATOM_BYTES);
+                mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u * BKS : (uint32_t)n_mt * PF_ATOM_BYTES);
                 const uint32_t a = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                if constexpr (BKS == 2) {  // (one-tile kernel) the two 64-column tiles of the stage's column block
+                    pf_tma_load_2d(a, &xmap, (kb0 + kb) * 2 * PF_BK, (int)m0, full(s));
+                    pf_tma_load_2d(a + pf_x_bytes(1), &xmap, (kb0 + kb) * 2 * PF_BK + PF_BK, (int)m0, full(s));
+                } else {
 #pragma unroll
-                for (int mt = 0; mt < MT; ++mt)
-                    if (mt < n_mt) pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
+                    for (int mt = 0; mt < MT; ++mt)
+                        if (mt < n_mt) pf_tma_load_2d(a + mt * PF_ATOM_BYTES, &xmap, (kb0 + kb) * PF_BK, (int)m0 + mt * PF_BM, full(s));
+                }
             }
         }
     } else if (warp <= NI) {
@@ -455,7 +485,37 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                     }
                     __syncwarp();
                 }
-                uint32_t s16 = sc2[buf];
+                if constexpr (AT && BKS == 2) {
+                    // a whole record: the two 64-column halves in turn, 32 packed pairs = 32 columns of this thread's lane each
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");  // (behind the wait for the stage)
+#pragma unroll
+                    for (int hb = 0; hb < 2; ++hb) {
+                        uint32_t sh = sc2[buf][hb];
+                        if (DT == 1) sh = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)sh))));
+                        const uint32_t sh2 = sh * 0x10001u;
+                        uint32_t wa[32];
+#pragma unroll
+                        for (int T2 = 0; T2 < 2; ++T2) {
+                            uint32_t w2[16];
+                            if (row_ok) {
+                                if (DT == 0) potl::pot_decode32<BITS, 4>(rec[buf], 2 * hb + T2, sh2, w2);
+                                else potl::pot_decode32_bf16<BITS, 4>(rec[buf], 2 * hb + T2, sh2, w2);
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 16; ++q) w2[q] = 0u;
+                            }
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) wa[16 * T2 + q] = w2[q];
+                        }
+                        pf_st32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(pf_at_ring_col0(MT) + 64 * s + 32 * hb), wa);
+                    }
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full(s));
+                    continue;
+                }
+                uint32_t s16 = sc2[buf][0];
                 if (DT == 1) s16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((uint16_t)s16))));
                 const uint32_t s2 = s16 * 0x10001u;  // scale pattern in both halves
                 if constexpr (AT) {
@@ -523,8 +583,10 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         item(tile, zsplit, splits);
         const int tail_index = tile - n_full;   // index of the tile among the split ones
         const int64_t rows_alloc = M < PF_BM * MT ? M : PF_BM * MT;  // token rows kept per tile in the workspace
-        constexpr int CH = (MT * PF_BM / 32) / NG;   // 32-column chunks per warp: the NG warps of a lane quarter share the tile's columns
-        static_assert(CH * NG * 32 == MT * PF_BM, "the epilogue warps must cover every token column");
+        // 32-column chunks per warp: the NG warps of a lane quarter share the tile's columns (the one-tile kernel holds at
+        // most PF_SMALL_TOKENS tokens: two chunks, whatever NG is)
+        constexpr int CH = MT == 1 ? 1 : (MT * PF_BM / 32) / NG;
+        static_assert(MT == 1 ? NG * 32 >= PF_SMALL_TOKENS : CH * NG * 32 == MT * PF_BM, "the epilogue warps must cover every token column");
 #pragma unroll
         for (int cc = 0; cc < CH; ++cc) {
             const int col = (part * CH + cc) * 32;
@@ -717,10 +779,10 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 4, 4, 2, 2, 1>, 4, 2);
         return run(pot_gemm_prefill_kernel<4, 4, 4, 2, 2, 1>, 4, 2);
     }
-    if (M <= PF_SMALL_TOKENS && prefill_weight_tile_in_tmem()) {  // twelve 8 KB stages of X, the A ring fills tensor memory
-        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
-        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
-        return run(pot_gemm_prefill_kernel<4, 12, 4, 2, 1, 0, 1>, 12, 1, 1, 4);
+    if (M <= PF_SMALL_TOKENS && prefill_weight_tile_in_tmem()) {  // six stages of a whole 128-column block (16 KB of X), three producer groups; the A ring fills tensor memory
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 3, 2, 1, 0, 1>, 6, 1, 1, 3);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 3, 2, 1, 0, 1>, 6, 1, 1, 3);
+        return run(pot_gemm_prefill_kernel<4, 6, 3, 2, 1, 0, 1>, 6, 1, 1, 3);
     }
     if (M <= PF_SMALL_TOKENS) {
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
