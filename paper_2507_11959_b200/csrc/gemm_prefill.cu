@@ -27,7 +27,8 @@
 // columns (see pf_issue_at).  The description above is the shared-memory-tile kernel, kept for the one-token-tile
 // variant and as a selectable alternative.
 // Batches of up to 64 tokens run a variant with one tile of M token rows (the TMA box holds exactly M rows, the MMA's
-// N is M rounded up to 16), eight 24 KB stages (twelve of 8 KB with the weight ring in tensor memory) and two TMA threads.
+// N is M rounded up to 16), eight 24 KB stages and two TMA threads; with the weight ring in tensor memory: six stages that
+// are whole 128-column blocks (two X tiles = 16 KB, 64 columns of weights, eight MMAs) and three producer groups.
 //
 // All mbarrier waits are bounded (see sync.cuh); a wait that gives up records a code and the CTA carries
 // on, so a lost transaction cannot hang the GPU.  Tensor memory is released on every path.
@@ -762,8 +763,8 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
                           (uint16_t*)Y, partial, counters, pl.tiles_m, pl.n_full, pl.splits, prefill_error_ptr());
     };
-    // two issuers, one CTA per SM; for batches of up to 64 tokens: one token tile, four producer groups, twelve 8 KB stages
-    // of X with the weight ring in tensor memory (eight 24 KB stages with the weight tile in shared memory)
+    // two issuers, one CTA per SM; for batches of up to 64 tokens: one token tile, three producer groups, six stages of a whole
+    // 128-column block with the weight ring in tensor memory (four groups, eight 24 KB stages with the tile in shared memory)
     if (dt == 1) {
         if (M <= PF_SMALL_TOKENS) {
             if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1, 1>, 8, 1);
