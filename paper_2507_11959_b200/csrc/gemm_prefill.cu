@@ -766,6 +766,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
     // two issuers, one CTA per SM; for batches of up to 64 tokens: one token tile, three producer groups, six stages of a whole
     // 128-column block with the weight ring in tensor memory (four groups, eight 24 KB stages with the tile in shared memory)
     if (dt == 1) {
+        if (M <= PF_SMALL_TOKENS && prefill_weight_tile_in_tmem()) {
+            if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 3, 2, 1, 1, 1>, 6, 1, 1, 3);
+            if (bits == 3) return run(pot_gemm_prefill_kernel<3, 6, 3, 2, 1, 1, 1>, 6, 1, 1, 3);
+            return run(pot_gemm_prefill_kernel<4, 6, 3, 2, 1, 1, 1>, 6, 1, 1, 3);
+        }
         if (M <= PF_SMALL_TOKENS) {
             if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1, 1>, 8, 1);
             if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1, 1>, 8, 1);
