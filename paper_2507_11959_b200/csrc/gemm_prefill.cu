@@ -594,7 +594,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
-            if (NI == 2 && !AT2) {                // add the second issuer's sums (odd K blocks) to the first's: a fixed order
+            if (NI == 2 && !AT2 && nkb > 1) {     // add the second issuer's sums (odd K blocks) to the first's: a fixed order
+                                                  // (an item of a single stage -- K = 128 with 128-column stages -- has none)
                 uint32_t v1[32];
                 pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)((AT ? PF_AT1_ACC_STRIDE : PF_BM * MT) + col), v1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");

@@ -17,9 +17,10 @@ def B():
 # (M, N, K).  M <= 64 runs the one-token-tile variant (eight stages, a TMA box of exactly M rows, two TMA threads), larger
 # M the 256-token tiles: one exact tile; ragged M and N with several K blocks; several tiles in both directions;
 # (300, ...) and (20, ...) run split-K; 129 tokens = a second token tile that holds one token; 64 / 65 tokens = either
-# side of the variant boundary; K = 1152 / 2048 = more K blocks than pipeline stages
+# side of the variant boundary; K = 1152 / 2048 = more K blocks than pipeline stages; K = 128 = a single stage (one-tile
+# kernel) or two (256-token kernel); 896 = seven column blocks, one more than the one-tile kernel's six stages
 SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20, 256, 4096), (129, 144, 640),
-          (64, 272, 1152), (9, 48, 2048), (65, 160, 1152)]
+          (64, 272, 1152), (9, 48, 2048), (65, 160, 1152), (17, 32, 128), (70, 16, 128), (48, 400, 896)]
 
 
 @pytest.fixture(params=["smem", "tmem"])
