@@ -123,6 +123,20 @@ def test_pot_gemm_fallback_matches_oracle(B, oracle, bits, M):
         assert ok and tight < 4.0, ("fallback", N, K, M, worst, tight)
 
 
+@pytest.mark.parametrize("M", [2, 4])
+def test_small_batch_with_activations_too_long_for_shared_memory(B, oracle, M):
+    """K = 28672: two tokens still fit in the streaming kernel's staging area (two token slots), four do not and are
+    read from global memory for every unit."""
+    bits, G, N, K = 3, 128, 32, 28672
+    c = PotCase(N, K, bits, G, dist="t5", seed=(4, 950))
+    X = acts(M, K, 951)
+    Y, A = oracle.matmul(c.packed, c.S, K, bits, G, X)
+    Yg = B.pot_gemm(c.tiled(), c.tiled_S(), K, bits, G, f16_dev(X), B.TILED)
+    ok, worst, tight = gate(bits_of(Yg), Y, A)
+    assert ok and tight < 4.0, (M, worst, tight)
+    assert B.pot_debug_errors() == (0, 0, 0)
+
+
 def test_gemv_with_activations_too_long_for_shared_memory(B, oracle):
     """K = 65536: the activation vector (128 KB) no longer fits the kernel's shared-memory staging area and is read
     from global memory instead -- PoT and uniform twin."""
