@@ -129,3 +129,35 @@ def test_weights_written_just_before_the_gemv_are_complete(oracle):
         y, _, _ = run(Ws[r], False)
         assert torch.equal(y, ref[r][0]), (it, r)
     assert B.pot_debug_errors() == (0, 0, 0)
+
+
+@pytest.mark.parametrize("M", [16, 200])
+def test_weights_written_just_before_the_tcgen05_gemm_are_complete(oracle, M):
+    """The same for the tcgen05 kernels (one-tile and 256-token variants), whose producers fetch their first codes and
+    scales even before the kernel's set-up."""
+    bits, G, N, K, R = 3, 128, 1024, 2048, 4
+    X = f16_dev(synth.activations(synth.rng_for(8, 400), M, K))
+    ws = B.new_workspace(B.pot_gemm_workspace_bytes(M, N, K, bits, G), DEV)
+    Ws = [f16_dev(synth.weights(synth.rng_for(8, 410 + r), N, K, "normal")) for r in range(R)]
+
+    def run(W, sync):
+        packed, S = B.pot_quantize_ref(W, bits, G, B.SCALE_TOP)
+        if sync:
+            torch.cuda.synchronize()
+        tiled = B.pot_repack(packed, K, bits, 0)
+        tS = B.pot_repack_scales(S, K, G, 0)
+        if sync:
+            torch.cuda.synchronize()
+        Y = B.pot_gemm(tiled, tS, K, bits, G, X, B.TILED, workspace=ws)
+        torch.cuda.synchronize()
+        return Y, packed, S
+
+    ref = [run(W, True) for W in Ws]
+    Yo, A = oracle.matmul(ref[0][1].cpu().numpy(), bits_of(ref[0][2]), K, bits, G, bits_of(X))
+    ok, worst, tight = gate(bits_of(ref[0][0]), Yo, A)
+    assert ok and tight < 4.0, (worst, tight)
+    for it in range(4 * R):
+        r = (3 * it) % R
+        Y, _, _ = run(Ws[r], False)
+        assert torch.equal(Y, ref[r][0]), (it, r)
+    assert B.pot_debug_errors() == (0, 0, 0)
