@@ -35,6 +35,7 @@
 #include <cuda.h>
 
 #include <cstdlib>
+#include <cstring>
 
 #include <type_traits>
 
@@ -60,9 +61,11 @@ __host__ __device__ constexpr int pf_x_bytes(int mt) { return mt == 1 ? PF_SMALL
 // (at = 1: the decoded weight tile lives in tensor memory, a stage of shared memory holds the X tiles only)
 // K sub-blocks of 64 columns per stage: two in the one-tile kernel with the weight ring in tensor memory (a stage is then a
 // whole 128-column block: half as many stage visits per byte for every role), one otherwise
-__host__ __device__ constexpr int pf_bks(int mt, int at) { return (mt == 1 && at) ? 2 : 1; }
-__host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0) { return pf_x_bytes(mt) * pf_bks(mt, at) + (at ? 0 : PF_ATOM_BYTES); }
-constexpr size_t pf_smem_bytes(int stages, int mt, int at = 0) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt, at) + 256 /*barriers*/; }
+// (wide = 1 asks for them in the 256-token kernel too: for a single wave of tiles, where the stage visits and not the tensor
+// pipe set the pace)
+__host__ __device__ constexpr int pf_bks(int mt, int at, int wide = 0) { return (at && (mt == 1 || wide)) ? 2 : 1; }
+__host__ __device__ constexpr int pf_stage_bytes(int mt, int at = 0, int wide = 0) { return pf_x_bytes(mt) * pf_bks(mt, at, wide) + (at ? 0 : PF_ATOM_BYTES); }
+constexpr size_t pf_smem_bytes(int stages, int mt, int at = 0, int wide = 0) { return 1024 /*align slack*/ + (size_t)stages * pf_stage_bytes(mt, at, wide) + 256 /*barriers*/; }
 constexpr int PF_AT_ACC_COLS = 256;   // at = 1, 256-token tiles: accumulator columns (token t of the tile = column t), then 32 columns per stage of A
 // at = 1, the one-tile kernel (up to 64 tokens): the two issuers' accumulators take 64 columns each, the A ring follows
 constexpr int PF_AT1_ACC_STRIDE = PF_SMALL_TOKENS;
@@ -166,7 +169,7 @@ __device__ __forceinline__ void pf_st32(uint32_t taddr, const uint32_t (&r)[32])
 // (A, from tensor memory: 128 weight rows x 64) by token tile J of the stage (B, 128 tokens, from shared memory) and
 // accumulates into columns 128 J .. 128 J + 127 -- the two issuers share the weight tile and never the accumulator, so
 // the order of the additions is fixed.  A stage is free again when every active issuer's MMAs on it have completed.
-template <int J, int PF_STAGES, int DT>
+template <int J, int PF_STAGES, int DT, int BKS = 1>
 __device__ __forceinline__ void pf_issue_at(uint32_t smem0, uint32_t bar0, uint32_t tmem_base, int nkb, int* err) {
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (PF_STAGES + s); };
@@ -174,8 +177,9 @@ __device__ __forceinline__ void pf_issue_at(uint32_t smem0, uint32_t bar0, uint3
     uint32_t blo[PF_STAGES];
 #pragma unroll
     for (int s = 0; s < PF_STAGES; ++s)
-        blo[s] = (uint32_t)pf_smem_desc(smem0 + (uint32_t)s * pf_stage_bytes(PF_MT, 1) + (uint32_t)J * PF_ATOM_BYTES);
+        blo[s] = (uint32_t)pf_smem_desc(smem0 + (uint32_t)s * pf_stage_bytes(PF_MT, 1, BKS == 2) + (uint32_t)J * PF_ATOM_BYTES);
     constexpr uint32_t desc_hi = (uint32_t)(PF_DESC_CONST >> 32);
+    constexpr uint32_t SLOT = 32u * BKS;   // tensor-memory columns of a stage's weights
     const uint32_t d0 = tmem_base + (uint32_t)(J * PF_BM);
     const uint32_t a0 = tmem_base + (uint32_t)PF_AT_ACC_COLS;
     const uint32_t idesc = pf_idesc(PF_BM, DT);
@@ -193,8 +197,9 @@ __device__ __forceinline__ void pf_issue_at(uint32_t smem0, uint32_t bar0, uint3
             if (kb + 1 < nkb) ready = mbar_test(full((s + 1) % PF_STAGES), s + 1 >= PF_STAGES ? ph ^ 1u : ph);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int ks = 0; ks < PF_BK / 16; ++ks)
-                pf_mma_ta(d0, a0 + (uint32_t)(32 * s + 8 * ks), blo[s] + (uint32_t)((ks * 32) >> 4), desc_hi, idesc,
+            for (int ks = 0; ks < BKS * (PF_BK / 16); ++ks)   // sub-block ks / 4: its X tiles follow the first sub-block's
+                pf_mma_ta(d0, a0 + SLOT * (uint32_t)s + (uint32_t)(8 * ks),
+                          blo[s] + (uint32_t)(((ks >> 2) * PF_MT * PF_ATOM_BYTES + (ks & 3) * 32) >> 4), desc_hi, idesc,
                           (s != 0 || ks != 0) ? 1u : (uint32_t)(kb0 != 0));
             pf_commit(empty(s));
         }
@@ -299,7 +304,7 @@ __device__ __forceinline__ void pf_issue(uint32_t smem0, uint32_t bar0, uint32_t
 // <bits, 6, 2, 2, 2, dt, 1>: 256 accumulator columns + 6 x 32 columns of A = 448 of the 512 columns.
 // NGP of the NG groups decode, the others only take part in the epilogue (measured slower than NGP = NG = 2 -- the
 // waiting groups poll the accumulator barrier through the whole main loop -- and not instantiated).
-template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0, int AT = 0, int NGP = NG>  // DT = 1: BF16 activations, weights and output
+template <int BITS, int PF_STAGES, int NG, int NI, int MT, int DT = 0, int AT = 0, int NGP = NG, int WIDE = 0>  // DT = 1: BF16 activations, weights and output
 __global__ void __launch_bounds__(pf_threads(NG, NI), 1)
 pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* __restrict__ packed,
                         const uint16_t* __restrict__ scales, int64_t N, int64_t K, int G, int64_t M,
@@ -310,8 +315,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     static_assert(AT == 0 || NI == 2, "the tensor-memory weight tile is built for two issuers");
     constexpr bool AT2 = AT && MT == 2;   // both issuers on every stage, one token tile each (else: alternate stages)
-    constexpr int BKS = pf_bks(MT, AT);   // 64-column sub-blocks per stage
-    constexpr int STAGE_BYTES = pf_stage_bytes(MT, AT);
+    constexpr int BKS = pf_bks(MT, AT, WIDE);   // 64-column sub-blocks per stage
+    constexpr int STAGE_BYTES = pf_stage_bytes(MT, AT, WIDE);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)PF_STAGES * STAGE_BYTES);
     // bars: full[S] (TMA bytes + one arrival per producer warp), empty[S], accum, then the tensor-memory base address
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PF_STAGES + 1);
@@ -323,7 +328,7 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
     constexpr int PROD_WARP0 = pf_prod_warp0(NI);
     constexpr int NPT = NG * 128;                       // producer / epilogue threads
     constexpr int TMEM_COLS = AT ? 512 : NI * PF_BN * MT;  // MT accumulators per issuer; AT: 256 accumulator columns + the A ring
-    static_assert((NGP % 2 == 0 || BKS == 2) && NGP <= NG && PF_STAGES % NI == 0 && PF_STAGES % NGP == 0,
+    static_assert((NGP % 2 == 0 || BKS == 2) && NGP <= NG && (AT2 || PF_STAGES % NI == 0) && PF_STAGES % NGP == 0,
                   "a group always decodes the same half of a column block; a stage buffer belongs to one issuer and one group");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items in launch order: the first n_full are whole output tiles; each of the remaining ("tail") tiles is cut
@@ -438,11 +443,18 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
                 ready = (kn < nkb && kn >= PF_STAGES) ? mbar_test(empty(kn % PF_STAGES), (uint32_t)((kn / PF_STAGES - 1) & 1)) : 0u;
                 // MT == 1 (M <= 64): the box holds exactly the M token rows -- the TMA unit spends time on every row of a
                 // box, in range or not; the rows of the tile that nothing writes belong to tokens that are never stored
-                mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u * BKS : (uint32_t)n_mt * PF_ATOM_BYTES);
+                mbar_expect_tx(full(s), MT == 1 ? (uint32_t)M * 128u * BKS : (uint32_t)n_mt * PF_ATOM_BYTES * BKS);
                 const uint32_t a = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                if constexpr (BKS == 2) {  // (one-tile kernel) the two 64-column tiles of the stage's column block
+                if constexpr (BKS == 2 && MT == 1) {  // (one-tile kernel) the two 64-column tiles of the stage's column block
                     pf_tma_load_2d(a, &xmap, (kb0 + kb) * 2 * PF_BK, (int)m0, full(s));
                     pf_tma_load_2d(a + pf_x_bytes(1), &xmap, (kb0 + kb) * 2 * PF_BK + PF_BK, (int)m0, full(s));
+                } else if constexpr (BKS == 2) {      // [sub-block][token tile] tiles of 16 KB
+#pragma unroll
+                    for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+                            if (mt < n_mt)
+                                pf_tma_load_2d(a + (sub * MT + mt) * PF_ATOM_BYTES, &xmap, ((kb0 + kb) * 2 + sub) * PF_BK, (int)m0 + mt * PF_BM, full(s));
                 } else {
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
@@ -454,8 +466,8 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         // ---------------- MMA issuers (one thread each) ------------------------------------------------
         if (lane == 0) {
             if constexpr (AT2) {
-                if (warp == 1) pf_issue_at<0, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
-                else if (n_mt == 2) pf_issue_at<1, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, err);
+                if (warp == 1) pf_issue_at<0, PF_STAGES, DT, BKS>(smem_u32(smem), bar0, tmem_base, nkb, err);
+                else if (n_mt == 2) pf_issue_at<1, PF_STAGES, DT, BKS>(smem_u32(smem), bar0, tmem_base, nkb, err);
             } else if constexpr (AT) {
                 if (warp == 1) pf_issue_at1<0, NI, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
                 else pf_issue_at1<NI - 1, NI, PF_STAGES, DT>(smem_u32(smem), bar0, tmem_base, nkb, n_tok, err);
@@ -586,11 +598,13 @@ pot_gemm_prefill_kernel(const __grid_constant__ CUtensorMap xmap, const uint4* _
         const int64_t rows_alloc = M < PF_BM * MT ? M : PF_BM * MT;  // token rows kept per tile in the workspace
         // 32-column chunks per warp: the NG warps of a lane quarter share the tile's columns (the one-tile kernel holds at
         // most PF_SMALL_TOKENS tokens: two chunks, whatever NG is)
-        constexpr int CH = MT == 1 ? 1 : (MT * PF_BM / 32) / NG;
-        static_assert(MT == 1 ? NG * 32 >= PF_SMALL_TOKENS : CH * NG * 32 == MT * PF_BM, "the epilogue warps must cover every token column");
+        // (chunks part, part + NG, ... of the tile's 32-column chunks; the one-tile kernel holds at most PF_SMALL_TOKENS tokens)
+        constexpr int NCH = MT == 1 ? PF_SMALL_TOKENS / 32 : MT * PF_BM / 32;
+        constexpr int CH = (NCH + NG - 1) / NG;
 #pragma unroll
         for (int cc = 0; cc < CH; ++cc) {
-            const int col = (part * CH + cc) * 32;
+            if (part + cc * NG >= NCH) break;
+            const int col = (part + cc * NG) * 32;
             if (m0 + col >= M) break;             // (warp-uniform) no token in these columns
             uint32_t v[32];
             pf_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
@@ -733,10 +747,16 @@ static int* prefill_error_ptr();
 // MMAs read their A operand there).  That takes a third of the traffic off shared memory, and a stage of shared memory
 // then holds X only, so six stages fit instead of four, and two producer groups keep up: measured 0.85 - 0.88 of the
 // cuBLAS burst figure on the six 70B points against 0.80 - 0.86 with the tile in shared memory (four stages, four
-// groups).  POT_PREFILL_WEIGHT_TILE = smem selects the shared-memory kernel (a diagnostic switch: the tests run both).
+// groups).  POT_PREFILL_WEIGHT_TILE = smem selects the shared-memory kernel (a diagnostic switch: the tests run all variants).
 static bool prefill_weight_tile_in_tmem() {
     const char* e = getenv("POT_PREFILL_WEIGHT_TILE");
     return !(e && e[0] == 's');
+}
+// POT_PREFILL_WEIGHT_TILE = tmem-narrow keeps the 256-token kernel on its 64-column stages even for a single wave of CTAs
+// (diagnostic: the tests run that kernel on small shapes this way)
+static bool prefill_wide_stages_allowed() {
+    const char* e = getenv("POT_PREFILL_WEIGHT_TILE");
+    return !(e && strcmp(e, "tmem-narrow") == 0);
 }
 
 pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t N, int64_t K, int bits, int group,
@@ -757,8 +777,8 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return POT_ERR_CUDA;
     const dim3 grid((unsigned)(pl.n_full + pl.n_tail * pl.splits));
-    auto run = [&](auto kernel, int stages, int mt, int at = 0, int ng = 4) -> pot_status_t {
-        const size_t smem = pf_smem_bytes(stages, mt, at);
+    auto run = [&](auto kernel, int stages, int mt, int at = 0, int ng = 4, int wide = 0) -> pot_status_t {
+        const size_t smem = pf_smem_bytes(stages, mt, at, wide);
         const dim3 block((unsigned)pf_threads(ng, 2));
         if (!allow_max_dynamic_smem(kernel)) return POT_ERR_CUDA;
         return launch_pdl(kernel, grid, block, smem, s, xmap, (const uint4*)packed, (const uint16_t*)scales, N, K, group, M,
@@ -776,6 +796,11 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
             if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1, 1>, 8, 1);
             if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1, 1>, 8, 1);
             return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1, 1>, 8, 1);
+        }
+        if (prefill_weight_tile_in_tmem() && grid.x <= (unsigned)kSmCount && prefill_wide_stages_allowed()) {
+            if (bits == 2) return run(pot_gemm_prefill_kernel<2, 3, 3, 2, 2, 1, 1, 3, 1>, 3, 2, 1, 3, 1);
+            if (bits == 3) return run(pot_gemm_prefill_kernel<3, 3, 3, 2, 2, 1, 1, 3, 1>, 3, 2, 1, 3, 1);
+            return run(pot_gemm_prefill_kernel<4, 3, 3, 2, 2, 1, 1, 3, 1>, 3, 2, 1, 3, 1);
         }
         if (prefill_weight_tile_in_tmem()) {
             if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 2, 2, 2, 1, 1>, 6, 2, 1, 2);
@@ -795,6 +820,15 @@ pot_status_t gemm_prefill_launch(const void* packed, const void* scales, int64_t
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 8, 4, 2, 1>, 8, 1);
         if (bits == 3) return run(pot_gemm_prefill_kernel<3, 8, 4, 2, 1>, 8, 1);
         return run(pot_gemm_prefill_kernel<4, 8, 4, 2, 1>, 8, 1);
+    }
+    // A single wave of CTAs (65 .. 256 tokens on decode-sized matrices) is paced by the stage visits, not by the tensor
+    // pipe: three stages of a whole 128-column block (64 KB of X, 64 columns of weights, three producer groups), as in the
+    // one-tile kernel (15360 x 5120 at 65 .. 128 tokens: 27.5 - 28.5 -> 22.2 - 23.1 us).
+    const bool one_wave = grid.x <= (unsigned)kSmCount && prefill_wide_stages_allowed();
+    if (prefill_weight_tile_in_tmem() && one_wave) {
+        if (bits == 2) return run(pot_gemm_prefill_kernel<2, 3, 3, 2, 2, 0, 1, 3, 1>, 3, 2, 1, 3, 1);
+        if (bits == 3) return run(pot_gemm_prefill_kernel<3, 3, 3, 2, 2, 0, 1, 3, 1>, 3, 2, 1, 3, 1);
+        return run(pot_gemm_prefill_kernel<4, 3, 3, 2, 2, 0, 1, 3, 1>, 3, 2, 1, 3, 1);
     }
     if (prefill_weight_tile_in_tmem()) {  // two producer groups, six stages (32 KB of X each), the A ring in tensor memory
         if (bits == 2) return run(pot_gemm_prefill_kernel<2, 6, 2, 2, 2, 0, 1>, 6, 2, 1, 2);

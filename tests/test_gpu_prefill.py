@@ -23,10 +23,11 @@ SHAPES = [(128, 128, 128), (200, 144, 384), (33, 16, 256), (300, 272, 1152), (20
           (64, 272, 1152), (9, 48, 2048), (65, 160, 1152), (17, 32, 128), (70, 16, 128), (48, 400, 896)]
 
 
-@pytest.fixture(params=["smem", "tmem"])
+@pytest.fixture(params=["smem", "tmem", "tmem-narrow"])
 def weight_tile(request, monkeypatch):
-    """The large-M kernel keeps the decoded weight tile in shared memory or in tensor memory (chosen by K in production):
-    the parity tests run both through the library's diagnostic switch."""
+    """The tcgen05 kernels keep the decoded weight tile in tensor memory (the default: a single wave of CTAs then runs
+    128-column stages; "tmem-narrow" keeps the 64-column stages that larger launches use) or in shared memory: the parity
+    tests run all three through the library's diagnostic switch."""
     monkeypatch.setenv("POT_PREFILL_WEIGHT_TILE", request.param)
     return request.param
 
